@@ -1,0 +1,378 @@
+/*
+ * FVAttn oracle: a plain, slow, fp64 CPU statement of what the sparse-routing
+ * frontend and the block-sparse attention compute.
+ *
+ * THIS IS TEST INFRASTRUCTURE.  Only the tests, the smoke check and the
+ * benchmark's cpu-baseline leg may call it.  It shares no code with the CUDA
+ * library, is never used as a fallback, and is deliberately untuned: every
+ * function takes the steps in the order the paper states them, one loop per
+ * step, no blocking or fusion.
+ *
+ * Passages followed (paper section / equation):
+ *   - Sec. 2.1: importance score s[h,i,j], binary block mask M[h,i,j]; only the
+ *     selected (query block, key block) pairs are evaluated.
+ *   - Sec. 2.1: Top-k keeps the k best key blocks; Top-p keeps the smallest set
+ *     whose cumulative normalised importance reaches p; FVAttn = Top-p with a
+ *     Top-k floor.
+ *   - Sec. 3.1: blocks come from a video-aware reorder of the token grid; block
+ *     similarities come from pooled Q/K; the same pass yields the per-head
+ *     density and the key-block importance order.
+ *   - Eq. 1: L_h = mean_i sum_j M[h,i,j].
+ *
+ * Readings taken where the paper is silent (each is listed in the design notes):
+ *   reorder = 3-D tiles in raster order (t, y, x; x fastest), tokens inside a tile
+ *   in the same raster order; pooling = arithmetic mean over the valid tokens of
+ *   a block; score = sm_scale * <qbar, kbar>; normalisation = softmax over all
+ *   key blocks of the row; sort by score descending, ties by lower block index;
+ *   the block that crosses p is kept (>=); p >= 1 keeps all; p <= 0 keeps one
+ *   before the floor; floor = integer block count clamped to nb; padded tokens
+ *   are zero rows, left out of pooling, masked as keys, zero as queries.
+ *
+ * Parity pins: every function here is pinned by tests/test_oracle_pins.py
+ * (closed forms, invariants, brute force, library routines).  The paper prints
+ * no worked numeric example for this path, so numeric parity with the paper's
+ * own implementation is unpinned; only the definitions are pinned.
+ *
+ * Inputs are bf16 bit patterns (uint16_t); all arithmetic is double.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+typedef struct {
+    int32_t T, Y, X;    /* latent grid */
+    int32_t tT, tY, tX; /* tile (block) shape */
+} ogrid_t;
+
+static double bf16_to_f64(uint16_t b) {
+    uint32_t u = ((uint32_t)b) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+static int32_t ceil_div(int32_t a, int32_t b) { return (a + b - 1) / b; }
+
+int32_t oracle_block_tokens(const ogrid_t* g) { return g->tT * g->tY * g->tX; }
+
+int32_t oracle_num_blocks(const ogrid_t* g) {
+    return ceil_div(g->T, g->tT) * ceil_div(g->Y, g->tY) * ceil_div(g->X, g->tX);
+}
+
+int64_t oracle_padded_tokens(const ogrid_t* g) {
+    return (int64_t)oracle_num_blocks(g) * oracle_block_tokens(g);
+}
+
+int32_t oracle_threads(void) {
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+/* Sec. 3.1 (reorder), tile reading: token n = (t*Y + y)*X + x goes to row
+ * blk*Bs + off with blk the raster index of its tile and off its raster
+ * index inside the tile. */
+static int64_t token_to_row(const ogrid_t* g, int32_t t, int32_t y, int32_t x) {
+    int32_t nY = ceil_div(g->Y, g->tY), nX = ceil_div(g->X, g->tX);
+    int64_t blk = ((int64_t)(t / g->tT) * nY + (y / g->tY)) * nX + (x / g->tX);
+    int64_t off = ((int64_t)(t % g->tT) * g->tY + (y % g->tY)) * g->tX + (x % g->tX);
+    return blk * oracle_block_tokens(g) + off;
+}
+
+/* pi[n] = reordered row of token n, n in raster order over (T, Y, X). */
+void oracle_permutation(const ogrid_t* g, int64_t* pi) {
+    for (int32_t t = 0; t < g->T; ++t)
+        for (int32_t y = 0; y < g->Y; ++y)
+            for (int32_t x = 0; x < g->X; ++x)
+                pi[((int64_t)t * g->Y + y) * g->X + x] = token_to_row(g, t, y, x);
+}
+
+/* valid[r] = 1 iff reordered row r is the image of a token. */
+void oracle_valid_rows(const ogrid_t* g, uint8_t* valid) {
+    int64_t n_pad = oracle_padded_tokens(g);
+    memset(valid, 0, (size_t)n_pad);
+    int64_t n = (int64_t)g->T * g->Y * g->X;
+    int64_t* pi = (int64_t*)malloc(sizeof(int64_t) * (size_t)n);
+    oracle_permutation(g, pi);
+    for (int64_t i = 0; i < n; ++i) valid[pi[i]] = 1;
+    free(pi);
+}
+
+/* src: [B, N, H, d] with element strides (sb, sn, sh), d contiguous.
+ * dst: [B, H, N_pad, d] dense; rows outside the image of pi are zero. */
+void oracle_reorder(const uint16_t* src, int32_t B, int32_t H, int32_t d, int64_t sb, int64_t sn,
+                    int64_t sh, const ogrid_t* g, uint16_t* dst) {
+    int64_t n = (int64_t)g->T * g->Y * g->X, n_pad = oracle_padded_tokens(g);
+    int64_t* pi = (int64_t*)malloc(sizeof(int64_t) * (size_t)n);
+    oracle_permutation(g, pi);
+    memset(dst, 0, sizeof(uint16_t) * (size_t)((int64_t)B * H * n_pad * d));
+    for (int32_t b = 0; b < B; ++b)
+        for (int32_t h = 0; h < H; ++h)
+            for (int64_t i = 0; i < n; ++i)
+                memcpy(dst + (((int64_t)b * H + h) * n_pad + pi[i]) * d, src + b * sb + i * sn + h * sh,
+                       sizeof(uint16_t) * (size_t)d);
+    free(pi);
+}
+
+/* out[n] = in[pi(n)]; pad rows are dropped.  dst has the token layout of
+ * oracle_reorder's src. */
+void oracle_inverse_reorder(const uint16_t* src_r, int32_t B, int32_t H, int32_t d, const ogrid_t* g,
+                            uint16_t* dst, int64_t sb, int64_t sn, int64_t sh) {
+    int64_t n = (int64_t)g->T * g->Y * g->X, n_pad = oracle_padded_tokens(g);
+    int64_t* pi = (int64_t*)malloc(sizeof(int64_t) * (size_t)n);
+    oracle_permutation(g, pi);
+    for (int32_t b = 0; b < B; ++b)
+        for (int32_t h = 0; h < H; ++h)
+            for (int64_t i = 0; i < n; ++i)
+                memcpy(dst + b * sb + i * sn + h * sh, src_r + (((int64_t)b * H + h) * n_pad + pi[i]) * d,
+                       sizeof(uint16_t) * (size_t)d);
+    free(pi);
+}
+
+/* Sec. 3.1 "pooled Q/K", mean reading: mean over the valid rows of each block.
+ * x_r: [BH, N_pad, d] bf16;  mean: [BH, nb, d] f64. */
+void oracle_pool(const uint16_t* x_r, int32_t BH, int32_t d, const ogrid_t* g, double* mean) {
+    int32_t nb = oracle_num_blocks(g), bs = oracle_block_tokens(g);
+    int64_t n_pad = oracle_padded_tokens(g);
+    uint8_t* valid = (uint8_t*)malloc((size_t)n_pad);
+    oracle_valid_rows(g, valid);
+#pragma omp parallel for collapse(2) schedule(static)
+    for (int32_t bh = 0; bh < BH; ++bh)
+        for (int32_t i = 0; i < nb; ++i) {
+            double* m = mean + ((int64_t)bh * nb + i) * d;
+            for (int32_t c = 0; c < d; ++c) m[c] = 0.0;
+            int32_t cnt = 0;
+            for (int32_t o = 0; o < bs; ++o) {
+                int64_t r = (int64_t)i * bs + o;
+                if (!valid[r]) continue;
+                const uint16_t* row = x_r + ((int64_t)bh * n_pad + r) * d;
+                for (int32_t c = 0; c < d; ++c) m[c] += bf16_to_f64(row[c]);
+                ++cnt;
+            }
+            for (int32_t c = 0; c < d; ++c) m[c] /= (double)cnt;
+        }
+    free(valid);
+}
+
+typedef struct {
+    double s;
+    int32_t j;
+} scored_t;
+
+/* score descending, ties by block index ascending */
+static int cmp_scored(const void* a, const void* b) {
+    const scored_t* x = (const scored_t*)a;
+    const scored_t* y = (const scored_t*)b;
+    if (x->s > y->s) return -1;
+    if (x->s < y->s) return 1;
+    return (x->j > y->j) - (x->j < y->j);
+}
+
+/*
+ * Routing (Sec. 2.1 Top-p with Top-k floor; Sec. 3.1 pooled similarities; Eq. 1).
+ * For every (bh, i):
+ *   s[j]   = sm_scale * <qbar[bh,i], kbar[bh,j]>
+ *   P[j]   = exp(s[j] - max s) / sum_j exp(s[j] - max s)
+ *   order  = blocks by s descending (ties: lower j)
+ *   c_p    = smallest m >= 1 with P_(1) + ... + P_(m) >= p   (nb if p >= 1 or never)
+ *   c      = max(c_p, min(k_floor, nb));  retained = first c of order
+ * Outputs:
+ *   mask_bits [BH, nb, ceil(nb/32)]  bit (j & 31) of word j >> 5
+ *   counts    [BH, nb]
+ *   idx       [BH, nb, nb]  first counts entries = retained j ascending, rest 0xFFFF
+ *   head_load [BH]          mean_i counts (Eq. 1)
+ *   order     [BH, nb, nb]  full importance order (may be NULL)
+ *   cum_at    [BH, nb]      cumulative mass after c_p blocks    (may be NULL)
+ *   cum_before[BH, nb]      cumulative mass after c_p - 1 blocks (may be NULL)
+ *   gap       [BH, nb]      (P_(c) - P_(c+1)) / P_(c), 1 if c == nb (may be NULL)
+ */
+void oracle_route(const uint16_t* q_r, const uint16_t* k_r, int32_t BH, int32_t d, const ogrid_t* g,
+                  double p, int32_t k_floor, double sm_scale, uint32_t* mask_bits, int32_t* counts,
+                  uint16_t* idx, double* head_load, uint16_t* order, double* cum_at, double* cum_before,
+                  double* gap) {
+    int32_t nb = oracle_num_blocks(g);
+    int32_t words = (nb + 31) / 32;
+    double* qbar = (double*)malloc(sizeof(double) * (size_t)BH * nb * d);
+    double* kbar = (double*)malloc(sizeof(double) * (size_t)BH * nb * d);
+    oracle_pool(q_r, BH, d, g, qbar);
+    oracle_pool(k_r, BH, d, g, kbar);
+
+#pragma omp parallel
+    {
+        scored_t* row = (scored_t*)malloc(sizeof(scored_t) * (size_t)nb);
+        double* prob = (double*)malloc(sizeof(double) * (size_t)nb);
+        uint8_t* keep = (uint8_t*)malloc((size_t)nb);
+#pragma omp for collapse(2) schedule(static)
+        for (int32_t bh = 0; bh < BH; ++bh)
+            for (int32_t i = 0; i < nb; ++i) {
+                const double* qv = qbar + ((int64_t)bh * nb + i) * d;
+                /* scores */
+                for (int32_t j = 0; j < nb; ++j) {
+                    const double* kv = kbar + ((int64_t)bh * nb + j) * d;
+                    double acc = 0.0;
+                    for (int32_t c = 0; c < d; ++c) acc += qv[c] * kv[c];
+                    row[j].s = sm_scale * acc;
+                    row[j].j = j;
+                }
+                /* softmax over the row */
+                double mx = row[0].s;
+                for (int32_t j = 1; j < nb; ++j)
+                    if (row[j].s > mx) mx = row[j].s;
+                double z = 0.0;
+                for (int32_t j = 0; j < nb; ++j) {
+                    prob[j] = exp(row[j].s - mx);
+                    z += prob[j];
+                }
+                for (int32_t j = 0; j < nb; ++j) prob[j] /= z;
+                /* descending order */
+                qsort(row, (size_t)nb, sizeof(scored_t), cmp_scored);
+                /* cumulative-mass cut */
+                int32_t cp = nb;
+                double cum = 0.0, at = 0.0, before = 0.0;
+                int found = 0;
+                for (int32_t m = 1; m <= nb; ++m) {
+                    double prev = cum;
+                    cum += prob[row[m - 1].j];
+                    if (!found && p < 1.0 && cum >= p) {
+                        cp = m;
+                        at = cum;
+                        before = prev;
+                        found = 1;
+                    }
+                }
+                if (!found) {
+                    at = cum;
+                    before = cum - prob[row[nb - 1].j];
+                }
+                /* floor */
+                int32_t fl = k_floor < nb ? k_floor : nb;
+                int32_t c = cp > fl ? cp : fl;
+                /* materialise */
+                memset(keep, 0, (size_t)nb);
+                for (int32_t m = 0; m < c; ++m) keep[row[m].j] = 1;
+                int64_t ri = (int64_t)bh * nb + i;
+                uint32_t* mb = mask_bits + ri * words;
+                for (int32_t w = 0; w < words; ++w) mb[w] = 0u;
+                uint16_t* ix = idx + ri * nb;
+                int32_t n_kept = 0;
+                for (int32_t j = 0; j < nb; ++j) {
+                    if (keep[j]) {
+                        mb[j >> 5] |= (1u << (j & 31));
+                        ix[n_kept++] = (uint16_t)j;
+                    }
+                }
+                for (int32_t m = n_kept; m < nb; ++m) ix[m] = 0xFFFFu;
+                counts[ri] = c;
+                if (order)
+                    for (int32_t m = 0; m < nb; ++m) order[ri * nb + m] = (uint16_t)row[m].j;
+                if (cum_at) cum_at[ri] = at;
+                if (cum_before) cum_before[ri] = before;
+                if (gap) {
+                    if (c >= nb) {
+                        gap[ri] = 1.0;
+                    } else {
+                        double pc = prob[row[c - 1].j], pn = prob[row[c].j];
+                        gap[ri] = pc > 0.0 ? (pc - pn) / pc : 0.0;
+                    }
+                }
+            }
+        free(row);
+        free(prob);
+        free(keep);
+    }
+    /* Eq. 1 */
+    if (head_load)
+        for (int32_t bh = 0; bh < BH; ++bh) {
+            double acc = 0.0;
+            for (int32_t i = 0; i < nb; ++i) acc += (double)counts[(int64_t)bh * nb + i];
+            head_load[bh] = acc / (double)nb;
+        }
+    free(qbar);
+    free(kbar);
+}
+
+/*
+ * Block-sparse attention (Sec. 2.1: only selected pairs are evaluated), written
+ * as the plain definition of masked softmax attention:
+ *   for query row r of block i (head bh), over keys r' in the retained blocks
+ *   that are valid tokens:
+ *     z[r'] = sm_scale * <Q[r], K[r']>;  w = softmax(z);  O[r] = sum w[r'] V[r']
+ *   padded query rows give 0.
+ * tiles == NULL: all (bh, i) tiles, out is [BH, N_pad, d].
+ * tiles != NULL: tiles[t] = bh * nb + i, out is [n_tiles, Bs, d].
+ */
+void oracle_sparse_attn(const uint16_t* q_r, const uint16_t* k_r, const uint16_t* v_r, const uint16_t* idx,
+                        const int32_t* counts, int32_t BH, int32_t d, const ogrid_t* g, double sm_scale,
+                        const int64_t* tiles, int64_t n_tiles, double* out) {
+    int32_t nb = oracle_num_blocks(g), bs = oracle_block_tokens(g);
+    int64_t n_pad = oracle_padded_tokens(g);
+    uint8_t* valid = (uint8_t*)malloc((size_t)n_pad);
+    oracle_valid_rows(g, valid);
+    int64_t total = tiles ? n_tiles : (int64_t)BH * nb;
+
+#pragma omp parallel
+    {
+        double* z = (double*)malloc(sizeof(double) * (size_t)n_pad);
+        double* qd = (double*)malloc(sizeof(double) * (size_t)d);
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t t = 0; t < total; ++t) {
+            int64_t tile = tiles ? tiles[t] : t;
+            int32_t bh = (int32_t)(tile / nb), i = (int32_t)(tile % nb);
+            const uint16_t* ix = idx + tile * nb;
+            int32_t c = counts[tile];
+            double* otile = tiles ? out + t * bs * d : out + ((int64_t)bh * n_pad + (int64_t)i * bs) * d;
+            for (int32_t o = 0; o < bs; ++o) {
+                int64_t r = (int64_t)i * bs + o;
+                double* orow = otile + (int64_t)o * d;
+                for (int32_t cc = 0; cc < d; ++cc) orow[cc] = 0.0;
+                if (!valid[r]) continue;
+                const uint16_t* qrow = q_r + ((int64_t)bh * n_pad + r) * d;
+                for (int32_t cc = 0; cc < d; ++cc) qd[cc] = bf16_to_f64(qrow[cc]);
+                /* logits over retained valid keys */
+                double mx = -INFINITY;
+                for (int32_t m = 0; m < c; ++m) {
+                    int64_t base = (int64_t)ix[m] * bs;
+                    for (int32_t oo = 0; oo < bs; ++oo) {
+                        int64_t rk = base + oo;
+                        if (!valid[rk]) continue;
+                        const uint16_t* krow = k_r + ((int64_t)bh * n_pad + rk) * d;
+                        double acc = 0.0;
+                        for (int32_t cc = 0; cc < d; ++cc) acc += qd[cc] * bf16_to_f64(krow[cc]);
+                        z[rk] = sm_scale * acc;
+                        if (z[rk] > mx) mx = z[rk];
+                    }
+                }
+                /* softmax weights and weighted sum of V */
+                double denom = 0.0;
+                for (int32_t m = 0; m < c; ++m) {
+                    int64_t base = (int64_t)ix[m] * bs;
+                    for (int32_t oo = 0; oo < bs; ++oo) {
+                        int64_t rk = base + oo;
+                        if (!valid[rk]) continue;
+                        z[rk] = exp(z[rk] - mx);
+                        denom += z[rk];
+                    }
+                }
+                for (int32_t m = 0; m < c; ++m) {
+                    int64_t base = (int64_t)ix[m] * bs;
+                    for (int32_t oo = 0; oo < bs; ++oo) {
+                        int64_t rk = base + oo;
+                        if (!valid[rk]) continue;
+                        double w = z[rk] / denom;
+                        const uint16_t* vrow = v_r + ((int64_t)bh * n_pad + rk) * d;
+                        for (int32_t cc = 0; cc < d; ++cc) orow[cc] += w * bf16_to_f64(vrow[cc]);
+                    }
+                }
+            }
+        }
+        free(z);
+        free(qd);
+    }
+    free(valid);
+}

@@ -1,0 +1,211 @@
+"""ctypes front end of the fp64 CPU oracle (``fvattn_oracle.c``).
+
+Test infrastructure only: the tests, the smoke check and the benchmark's
+cpu-baseline leg call this; the CUDA library never does and shares no code
+with it.  Tensors cross as numpy arrays: bf16 data as ``uint16`` bit patterns,
+results as ``float64`` / integer arrays.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "fvattn_oracle.c")
+_LIB = os.path.join(_HERE, "libfvattn_oracle.so")
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (portable flags: the .so may run on another host)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-std=c11", "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+class _Grid(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("T", "Y", "X", "tT", "tY", "tX")]
+
+
+@dataclass(frozen=True)
+class Grid:
+    """Latent grid (T, Y, X) and tile (block) shape (tT, tY, tX)."""
+
+    T: int
+    Y: int
+    X: int
+    tT: int
+    tY: int
+    tX: int
+
+    def c(self) -> _Grid:
+        return _Grid(self.T, self.Y, self.X, self.tT, self.tY, self.tX)
+
+    @property
+    def tokens(self) -> int:
+        return self.T * self.Y * self.X
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        L.oracle_num_blocks.restype = ctypes.c_int32
+        L.oracle_block_tokens.restype = ctypes.c_int32
+        L.oracle_padded_tokens.restype = ctypes.c_int64
+        L.oracle_threads.restype = ctypes.c_int32
+        _lib = L
+    return _lib
+
+
+def _p(a: np.ndarray | None):
+    if a is None:
+        return ctypes.c_void_p(0)
+    assert a.flags["C_CONTIGUOUS"]
+    return ctypes.c_void_p(a.ctypes.data)
+
+
+def _u16(a: np.ndarray) -> np.ndarray:
+    assert a.dtype == np.uint16, a.dtype
+    return np.ascontiguousarray(a)
+
+
+def threads() -> int:
+    return int(lib().oracle_threads())
+
+
+def num_blocks(g: Grid) -> int:
+    return int(lib().oracle_num_blocks(ctypes.byref(g.c())))
+
+
+def block_tokens(g: Grid) -> int:
+    return int(lib().oracle_block_tokens(ctypes.byref(g.c())))
+
+
+def padded_tokens(g: Grid) -> int:
+    return int(lib().oracle_padded_tokens(ctypes.byref(g.c())))
+
+
+def permutation(g: Grid) -> np.ndarray:
+    """pi[n] = reordered row of token n (raster order over T, Y, X)."""
+    pi = np.empty(g.tokens, dtype=np.int64)
+    lib().oracle_permutation(ctypes.byref(g.c()), _p(pi))
+    return pi
+
+
+def valid_rows(g: Grid) -> np.ndarray:
+    v = np.empty(padded_tokens(g), dtype=np.uint8)
+    lib().oracle_valid_rows(ctypes.byref(g.c()), _p(v))
+    return v
+
+
+def reorder(x: np.ndarray, g: Grid) -> np.ndarray:
+    """x: [B, N, H, d] uint16 (bf16 bits), dense -> [B, H, N_pad, d]."""
+    x = _u16(x)
+    B, N, H, d = x.shape
+    assert N == g.tokens
+    out = np.empty((B, H, padded_tokens(g), d), dtype=np.uint16)
+    lib().oracle_reorder(_p(x), ctypes.c_int32(B), ctypes.c_int32(H), ctypes.c_int32(d),
+                         ctypes.c_int64(N * H * d), ctypes.c_int64(H * d), ctypes.c_int64(d),
+                         ctypes.byref(g.c()), _p(out))
+    return out
+
+
+def inverse_reorder(x_r: np.ndarray, g: Grid) -> np.ndarray:
+    """x_r: [B, H, N_pad, d] uint16 -> [B, N, H, d] (pad rows dropped)."""
+    x_r = _u16(x_r)
+    B, H, n_pad, d = x_r.shape
+    assert n_pad == padded_tokens(g)
+    N = g.tokens
+    out = np.empty((B, N, H, d), dtype=np.uint16)
+    lib().oracle_inverse_reorder(_p(x_r), ctypes.c_int32(B), ctypes.c_int32(H), ctypes.c_int32(d),
+                                 ctypes.byref(g.c()), _p(out), ctypes.c_int64(N * H * d),
+                                 ctypes.c_int64(H * d), ctypes.c_int64(d))
+    return out
+
+
+def pool(x_r: np.ndarray, g: Grid) -> np.ndarray:
+    """x_r: [BH, N_pad, d] uint16 -> block means [BH, nb, d] float64."""
+    x_r = _u16(x_r)
+    BH, n_pad, d = x_r.shape
+    assert n_pad == padded_tokens(g)
+    out = np.empty((BH, num_blocks(g), d), dtype=np.float64)
+    lib().oracle_pool(_p(x_r), ctypes.c_int32(BH), ctypes.c_int32(d), ctypes.byref(g.c()), _p(out))
+    return out
+
+
+@dataclass
+class RouteResult:
+    mask_bits: np.ndarray   # [BH, nb, ceil(nb/32)] uint32
+    counts: np.ndarray      # [BH, nb] int32
+    idx: np.ndarray         # [BH, nb, nb] uint16, first counts entries ascending
+    head_load: np.ndarray   # [BH] float64 (Eq. 1)
+    order: np.ndarray | None        # [BH, nb, nb] uint16 importance order
+    cum_at: np.ndarray      # [BH, nb] mass after c_p blocks
+    cum_before: np.ndarray  # [BH, nb] mass after c_p - 1 blocks
+    gap: np.ndarray         # [BH, nb] relative gap last kept / first dropped
+
+    def mask_bool(self) -> np.ndarray:
+        """[BH, nb, nb] boolean expansion of mask_bits."""
+        BH, nb, words = self.mask_bits.shape
+        j = np.arange(nb)
+        return ((self.mask_bits[:, :, j >> 5] >> (j & 31).astype(np.uint32)) & 1).astype(bool)
+
+
+def route(q_r: np.ndarray, k_r: np.ndarray, g: Grid, p: float, k_floor: int, sm_scale: float,
+          want_order: bool = False) -> RouteResult:
+    """q_r, k_r: [BH, N_pad, d] uint16."""
+    q_r, k_r = _u16(q_r), _u16(k_r)
+    BH, n_pad, d = q_r.shape
+    assert k_r.shape == q_r.shape and n_pad == padded_tokens(g)
+    nb = num_blocks(g)
+    words = (nb + 31) // 32
+    res = RouteResult(
+        mask_bits=np.empty((BH, nb, words), dtype=np.uint32),
+        counts=np.empty((BH, nb), dtype=np.int32),
+        idx=np.empty((BH, nb, nb), dtype=np.uint16),
+        head_load=np.empty((BH,), dtype=np.float64),
+        order=np.empty((BH, nb, nb), dtype=np.uint16) if want_order else None,
+        cum_at=np.empty((BH, nb), dtype=np.float64),
+        cum_before=np.empty((BH, nb), dtype=np.float64),
+        gap=np.empty((BH, nb), dtype=np.float64),
+    )
+    lib().oracle_route(_p(q_r), _p(k_r), ctypes.c_int32(BH), ctypes.c_int32(d), ctypes.byref(g.c()),
+                       ctypes.c_double(p), ctypes.c_int32(k_floor), ctypes.c_double(sm_scale),
+                       _p(res.mask_bits), _p(res.counts), _p(res.idx), _p(res.head_load), _p(res.order),
+                       _p(res.cum_at), _p(res.cum_before), _p(res.gap))
+    return res
+
+
+def sparse_attn(q_r: np.ndarray, k_r: np.ndarray, v_r: np.ndarray, idx: np.ndarray, counts: np.ndarray,
+                g: Grid, sm_scale: float, tiles: np.ndarray | None = None) -> np.ndarray:
+    """Masked softmax attention over the retained blocks.
+
+    q_r, k_r, v_r: [BH, N_pad, d] uint16; idx [BH, nb, nb] uint16; counts [BH, nb] int32.
+    tiles None -> [BH, N_pad, d] float64; else tiles[t] = bh * nb + i -> [n_tiles, Bs, d].
+    """
+    q_r, k_r, v_r = _u16(q_r), _u16(k_r), _u16(v_r)
+    BH, n_pad, d = q_r.shape
+    nb, bs = num_blocks(g), block_tokens(g)
+    assert n_pad == padded_tokens(g) and k_r.shape == q_r.shape and v_r.shape == q_r.shape
+    idx = np.ascontiguousarray(idx, dtype=np.uint16)
+    counts = np.ascontiguousarray(counts, dtype=np.int32)
+    assert idx.shape == (BH, nb, nb) and counts.shape == (BH, nb)
+    if tiles is None:
+        out = np.empty((BH, n_pad, d), dtype=np.float64)
+        n_tiles = 0
+    else:
+        tiles = np.ascontiguousarray(tiles, dtype=np.int64)
+        n_tiles = tiles.shape[0]
+        out = np.empty((n_tiles, bs, d), dtype=np.float64)
+    lib().oracle_sparse_attn(_p(q_r), _p(k_r), _p(v_r), _p(idx), _p(counts), ctypes.c_int32(BH),
+                             ctypes.c_int32(d), ctypes.byref(g.c()), ctypes.c_double(sm_scale), _p(tiles),
+                             ctypes.c_int64(n_tiles), _p(out))
+    return out

@@ -1,0 +1,330 @@
+"""Pins for the CPU oracle: closed forms, invariants, brute force and library routines.
+
+The paper prints no worked numeric example for routing or attention, so every pin here is
+something the definitions (Sec. 2.1, Sec. 3.1, Eq. 1) or plain mathematics fix.  Each pin is
+computed by a route that does not go through the oracle's own arithmetic.
+"""
+import itertools
+import json
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import fvattn_oracle as O
+from paper_2607_16190_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def f32_to_bf16_bits(a: np.ndarray) -> np.ndarray:
+    return synth.bf16_bits(torch.from_numpy(np.asarray(a, dtype=np.float32)).to(torch.bfloat16))
+
+
+def bits_to_f64(a: np.ndarray) -> np.ndarray:
+    return synth.bits_to_bf16(a).to(torch.float64).numpy()
+
+
+def tiled_by_reshape(x: np.ndarray, g: O.Grid) -> np.ndarray:
+    """Independent statement of the 3-D tile reorder: pad the grid, split every axis into
+    (tile index, offset), bring the tile indices to the front.  x: [N, ...] -> [N_pad, ...]."""
+    T, Y, X, tT, tY, tX = g.T, g.Y, g.X, g.tT, g.tY, g.tX
+    nT, nY, nX = -(-T // tT), -(-Y // tY), -(-X // tX)
+    rest = x.shape[1:]
+    vol = np.zeros((nT * tT, nY * tY, nX * tX) + rest, dtype=x.dtype)
+    vol[:T, :Y, :X] = x.reshape((T, Y, X) + rest)
+    vol = vol.reshape((nT, tT, nY, tY, nX, tX) + rest)
+    perm = (0, 2, 4, 1, 3, 5) + tuple(range(6, 6 + len(rest)))
+    return vol.transpose(perm).reshape((nT * tT * nY * tY * nX * tX,) + rest)
+
+
+GRIDS = [
+    O.Grid(4, 8, 8, 1, 8, 8),
+    O.Grid(8, 16, 16, 2, 8, 8),
+    O.Grid(3, 5, 7, 2, 4, 4),        # ragged on every axis
+    O.Grid(2, 6, 20, 1, 8, 16),      # ragged y and x like the 480p case
+]
+
+
+# ---------------------------------------------------------------- reorder (Sec. 3.1)
+@pytest.mark.parametrize("g", GRIDS)
+def test_permutation_is_bijection_onto_valid_rows(g):
+    pi = O.permutation(g)
+    valid = O.valid_rows(g)
+    assert len(np.unique(pi)) == g.tokens
+    assert pi.min() >= 0 and pi.max() < O.padded_tokens(g)
+    assert valid.sum() == g.tokens
+    assert valid[pi].all()
+    assert pi[0] == 0                                   # token (0,0,0) opens block 0
+    last_block = pi[-1] // O.block_tokens(g)
+    assert last_block == O.num_blocks(g) - 1            # last token lands in the last block
+    # every block holds at least one token (padding is below one tile per axis)
+    assert valid.reshape(O.num_blocks(g), O.block_tokens(g)).any(axis=1).all()
+
+
+@pytest.mark.parametrize("g", GRIDS)
+def test_reorder_matches_reshape_formulation_and_inverts(g):
+    rng = np.random.default_rng(0)
+    B, H, d = 2, 3, 8
+    x = rng.integers(1, 2**16, size=(B, g.tokens, H, d), dtype=np.uint16)
+    x_r = O.reorder(x, g)
+    for b in range(B):
+        want = tiled_by_reshape(x[b], g)                # [N_pad, H, d]
+        np.testing.assert_array_equal(x_r[b], want.transpose(1, 0, 2))
+    valid = O.valid_rows(g).astype(bool)
+    assert (x_r[:, :, ~valid, :] == 0).all()            # pads are zero
+    np.testing.assert_array_equal(O.inverse_reorder(x_r, g), x)   # bit-for-bit identity
+
+
+def test_block_count_closed_form():
+    assert O.num_blocks(O.Grid(21, 45, 80, 1, 8, 16)) == 21 * 6 * 5 == 630
+    assert O.padded_tokens(O.Grid(21, 45, 80, 1, 8, 16)) == 80640
+    assert O.num_blocks(O.Grid(21, 30, 52, 1, 8, 16)) == 21 * 4 * 4 == 336
+    assert O.padded_tokens(O.Grid(21, 30, 52, 1, 8, 16)) == 43008
+
+
+# ---------------------------------------------------------------- pooling (Sec. 3.1)
+@pytest.mark.parametrize("g", GRIDS)
+def test_pool_constant_per_block_gives_the_constant(g):
+    """Mean over VALID tokens: an edge block with few valid rows still returns its constant
+    (dividing by the block size instead would scale it down)."""
+    nb, bs, d = O.num_blocks(g), O.block_tokens(g), 4
+    const = np.arange(1, nb + 1, dtype=np.float32)[:, None] * np.array([1, -1, 0.5, 2], np.float32)
+    valid = O.valid_rows(g).astype(bool)
+    rows = np.repeat(const, bs, axis=0)                 # [N_pad, d]
+    rows[~valid] = 0
+    mean = O.pool(f32_to_bf16_bits(rows)[None], g)[0]
+    np.testing.assert_allclose(mean, bits_to_f64(f32_to_bf16_bits(const)), rtol=0, atol=1e-12)
+
+
+@pytest.mark.parametrize("g", GRIDS)
+def test_pool_matches_numpy_masked_mean(g):
+    rng = np.random.default_rng(1)
+    d = 16
+    x = f32_to_bf16_bits(rng.standard_normal((1, g.tokens, 2, d)))
+    x_r = O.reorder(x, g)[0]                            # [H, N_pad, d]
+    nb, bs = O.num_blocks(g), O.block_tokens(g)
+    valid = O.valid_rows(g).reshape(nb, bs).astype(np.float64)
+    xf = bits_to_f64(x_r).reshape(2, nb, bs, d)
+    want = (xf * valid[None, :, :, None]).sum(2) / valid.sum(1)[None, :, None]
+    np.testing.assert_allclose(O.pool(x_r, g), want, rtol=1e-13, atol=1e-13)
+
+
+# ---------------------------------------------------------------- routing (Sec. 2.1)
+def _routing_inputs(name, seed_shift=0):
+    cfg = synth.CONFIGS[name]
+    cfg = cfg.with_(seed=cfg.seed + seed_shift)
+    q, k, v, _ = synth.make_qkv(cfg)
+    g = O.Grid(*cfg.grid, *cfg.tile)
+    q_r, k_r, v_r = (O.reorder(synth.bf16_bits(t), g)[0] for t in (q, k, v))
+    return cfg, g, q_r, k_r, v_r
+
+
+def _independent_probs(q_r, k_r, g, sm_scale):
+    """Row softmax of the block scores via numpy/torch primitives on numpy masked means."""
+    nb, bs = O.num_blocks(g), O.block_tokens(g)
+    valid = O.valid_rows(g).reshape(nb, bs).astype(np.float64)
+    H, _, d = q_r.shape
+
+    def mean(x):
+        xf = bits_to_f64(x).reshape(H, nb, bs, d)
+        return (xf * valid[None, :, :, None]).sum(2) / valid.sum(1)[None, :, None]
+
+    s = torch.from_numpy(np.einsum("hid,hjd->hij", mean(q_r), mean(k_r)) * sm_scale)
+    return s.numpy(), torch.softmax(s, dim=-1).numpy()
+
+
+def test_zero_queries_give_uniform_rows_and_ceil_count():
+    """Q = 0 => every score is 0 => P = 1/nb; with nb = 16 and p = 0.9 the cut keeps
+    ceil(0.9 * 16) = 15 blocks, and the index tie-break makes them blocks 0..14."""
+    cfg, g, q_r, k_r, _ = _routing_inputs("small")
+    q0 = np.zeros_like(q_r)
+    res = O.route(q0, k_r, g, 0.9, 2, cfg.sm_scale, want_order=True)
+    nb = O.num_blocks(g)
+    assert nb == 16
+    assert (res.counts == 15).all()
+    assert (res.idx[:, :, :15] == np.arange(15)).all() and (res.idx[:, :, 15] == 0xFFFF).all()
+    assert (res.order == np.arange(16)).all()
+    np.testing.assert_allclose(res.cum_at, 15 / 16, atol=1e-12)
+    np.testing.assert_allclose(res.cum_before, 14 / 16, atol=1e-12)
+    assert (res.mask_bits == 0x7FFF).all()
+
+
+@pytest.mark.parametrize("name,p", [("tiny", 0.9), ("small", 0.9), ("small", 0.5), ("small", 0.99)])
+def test_retained_mass_reaches_p_and_set_is_minimal(name, p):
+    cfg, g, q_r, k_r, _ = _routing_inputs(name)
+    res = O.route(q_r, k_r, g, p, cfg.k_floor, cfg.sm_scale, want_order=True)
+    _, P = _independent_probs(q_r, k_r, g, cfg.sm_scale)
+    M = res.mask_bool()
+    mass = (P * M).sum(-1)
+    assert (mass >= p - 1e-12).all()                      # reaches p
+    assert (M.sum(-1) == res.counts).all()
+    nb = O.num_blocks(g)
+    fl = min(cfg.k_floor, nb)
+    # minimality: above the floor, dropping the least important kept block falls below p
+    for h, i in zip(*np.nonzero(res.counts > fl)):
+        kept = np.nonzero(M[h, i])[0]
+        weakest = kept[np.argmin(P[h, i, kept])]
+        assert mass[h, i] - P[h, i, weakest] < p + 1e-12
+    # retained blocks are the top-c by score: no dropped block outranks a kept one
+    for h in range(M.shape[0]):
+        for i in range(nb):
+            if res.counts[h, i] < nb:
+                assert P[h, i][M[h, i]].min() >= P[h, i][~M[h, i]].max()
+    np.testing.assert_allclose(res.cum_at, np.where(res.cum_at > 0, res.cum_at, 0))
+    reached = res.counts > fl
+    np.testing.assert_allclose(mass[reached], res.cum_at[reached], atol=1e-12)
+
+
+def test_top_p_is_the_smallest_set_brute_force():
+    """nb = 4: enumerate all subsets; the smallest cardinality reaching p must equal the
+    oracle's count (floor 1), for several p."""
+    cfg, g, q_r, k_r, _ = _routing_inputs("tiny")
+    _, P = _independent_probs(q_r, k_r, g, cfg.sm_scale)
+    nb = O.num_blocks(g)
+    assert nb == 4
+    for p in (0.3, 0.6, 0.9, 0.97):
+        res = O.route(q_r, k_r, g, p, 1, cfg.sm_scale)
+        for h in range(P.shape[0]):
+            for i in range(nb):
+                best = min(len(sub) for r in range(1, nb + 1) for sub in itertools.combinations(range(nb), r)
+                           if P[h, i, list(sub)].sum() >= p)
+                assert res.counts[h, i] == best, (p, h, i)
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_p_to_zero_keeps_exactly_the_floor_and_equals_library_topk(name):
+    cfg, g, q_r, k_r, _ = _routing_inputs(name)
+    nb = O.num_blocks(g)
+    for k_floor in (1, 2, 3):
+        for p in (0.0, 1e-12):
+            res = O.route(q_r, k_r, g, p, k_floor, cfg.sm_scale)
+            assert (res.counts == min(k_floor, nb)).all()
+            s, _ = _independent_probs(q_r, k_r, g, cfg.sm_scale)
+            top = torch.topk(torch.from_numpy(s), min(k_floor, nb), dim=-1).indices.numpy()
+            np.testing.assert_array_equal(res.idx[:, :, :min(k_floor, nb)], np.sort(top, -1))
+    # floor above nb clamps to nb
+    res = O.route(q_r, k_r, g, 0.0, nb + 5, cfg.sm_scale)
+    assert (res.counts == nb).all()
+
+
+@pytest.mark.parametrize("name", ["tiny", "small"])
+def test_p_one_keeps_everything(name):
+    cfg, g, q_r, k_r, _ = _routing_inputs(name)
+    nb = O.num_blocks(g)
+    res = O.route(q_r, k_r, g, 1.0, cfg.k_floor, cfg.sm_scale)
+    assert (res.counts == nb).all() and res.mask_bool().all()
+    assert (res.idx == np.arange(nb)).all()
+
+
+def test_importance_order_is_a_library_argsort():
+    cfg, g, q_r, k_r, _ = _routing_inputs("small")
+    res = O.route(q_r, k_r, g, 0.9, 2, cfg.sm_scale, want_order=True)
+    s, _ = _independent_probs(q_r, k_r, g, cfg.sm_scale)
+    want = np.argsort(-s, axis=-1, kind="stable")
+    np.testing.assert_array_equal(res.order, want)
+
+
+def test_head_load_is_eq1():
+    cfg, g, q_r, k_r, _ = _routing_inputs("small")
+    res = O.route(q_r, k_r, g, 0.9, 2, cfg.sm_scale)
+    nb = O.num_blocks(g)
+    np.testing.assert_allclose(res.head_load, res.counts.mean(-1), rtol=1e-15)
+    popcount = sum(bin(int(w)).count("1") for w in res.mask_bits.ravel())
+    assert round(float(res.head_load.sum() * nb)) == popcount
+
+
+def test_hand_worked_rows():
+    """Rows whose probabilities are powers of two by construction (see the fixture)."""
+    with open(os.path.join(GOLDEN, "hand_worked_routing.json")) as f:
+        fx = json.load(f)
+    g = O.Grid(*fx["grid"], *fx["tile"])
+    nb, bs, d = O.num_blocks(g), O.block_tokens(g), fx["d"]
+    assert nb == 4
+    # block means: qbar_i = e_0 * a_i ; kbar_j = e_0 * b_j  => score = sm_scale * a_i * b_j
+    a, b = fx["q_block_value"], fx["k_block_value"]
+    q = np.zeros((1, nb * bs, d), np.float32)
+    k = np.zeros((1, nb * bs, d), np.float32)
+    for blk in range(nb):
+        q[0, blk * bs:(blk + 1) * bs, 0] = a[blk]
+        k[0, blk * bs:(blk + 1) * bs, 0] = b[blk]
+    for case in fx["cases"]:
+        res = O.route(f32_to_bf16_bits(q), f32_to_bf16_bits(k), g, case["p"], case["k_floor"],
+                      fx["sm_scale"], want_order=True)
+        assert res.counts[0].tolist() == case["counts"], case
+        for i, kept in enumerate(case["kept"]):
+            assert res.idx[0, i, :len(kept)].tolist() == kept, (case, i)
+
+
+# ---------------------------------------------------------------- attention (Sec. 2.1)
+def _dense_attention_tokens(q, k, v, sm_scale):
+    """Brute-force softmax attention on the ORIGINAL token order: q,k,v [N, H, d] f64."""
+    z = torch.einsum("nhd,mhd->hnm", q, k) * sm_scale
+    w = torch.softmax(z, dim=-1)
+    return torch.einsum("hnm,mhd->nhd", w, v)
+
+
+@pytest.mark.parametrize("name,tile2", [("tiny", (2, 4, 8)), ("small", (1, 16, 8))])
+def test_p_one_equals_dense_attention_and_is_tile_invariant(name, tile2):
+    cfg = synth.CONFIGS[name]
+    q, k, v, _ = synth.make_qkv(cfg)
+    want = _dense_attention_tokens(q[0].double(), k[0].double(), v[0].double(), cfg.sm_scale).numpy()
+    outs = []
+    for tile in (cfg.tile, tile2):
+        g = O.Grid(*cfg.grid, *tile)
+        q_r, k_r, v_r = (O.reorder(synth.bf16_bits(t), g)[0] for t in (q, k, v))
+        res = O.route(q_r, k_r, g, 1.0, cfg.k_floor, cfg.sm_scale)
+        o_r = O.sparse_attn(q_r, k_r, v_r, res.idx, res.counts, g, cfg.sm_scale)   # [H, N_pad, d]
+        o = o_r[:, O.permutation(g), :].transpose(1, 0, 2)                          # [N, H, d]
+        outs.append(o)
+        np.testing.assert_allclose(o, want, rtol=1e-10, atol=1e-12)
+    np.testing.assert_allclose(outs[0], outs[1], rtol=1e-10, atol=1e-12)
+
+
+@pytest.mark.parametrize("gridspec", [("tiny", None), ("small", None), ("small", (7, 13, 11))])
+def test_masked_attention_equals_library_sdpa_with_token_mask(gridspec):
+    """Expand the block mask to a boolean token mask (padded keys off) and call torch's
+    scaled_dot_product_attention in fp64 on the CPU."""
+    name, grid = gridspec
+    cfg = synth.CONFIGS[name]
+    if grid is not None:
+        cfg = cfg.with_(grid=grid, seed=11)
+    q, k, v, _ = synth.make_qkv(cfg)
+    g = O.Grid(*cfg.grid, *cfg.tile)
+    q_r, k_r, v_r = (O.reorder(synth.bf16_bits(t), g)[0] for t in (q, k, v))
+    res = O.route(q_r, k_r, g, 0.6, 1, cfg.sm_scale)
+    assert not res.mask_bool().all()
+    o_r = O.sparse_attn(q_r, k_r, v_r, res.idx, res.counts, g, cfg.sm_scale)
+    bs = O.block_tokens(g)
+    valid = torch.from_numpy(O.valid_rows(g).astype(bool))
+    tok_mask = torch.from_numpy(res.mask_bool()).repeat_interleave(bs, 1).repeat_interleave(bs, 2)
+    tok_mask = tok_mask & valid[None, None, :]
+    qf, kf, vf = (torch.from_numpy(bits_to_f64(t)) for t in (q_r, k_r, v_r))
+    want = torch.nn.functional.scaled_dot_product_attention(
+        qf[None], kf[None], vf[None], attn_mask=tok_mask[None], scale=cfg.sm_scale)[0]
+    want = torch.where(valid[None, :, None], want, torch.zeros_like(want))
+    np.testing.assert_allclose(o_r, want.numpy(), rtol=1e-9, atol=1e-12)
+    # sampled-tile form returns the same rows
+    nb = O.num_blocks(g)
+    tiles = np.array([0, nb - 1, nb + 1, res.counts.size - 1], dtype=np.int64)
+    sub = O.sparse_attn(q_r, k_r, v_r, res.idx, res.counts, g, cfg.sm_scale, tiles=tiles)
+    full = o_r.reshape(-1, nb, bs, cfg.d).reshape(-1, bs, cfg.d)
+    np.testing.assert_array_equal(sub, full[tiles])
+
+
+def test_single_retained_block_is_plain_attention_over_that_block():
+    cfg, g, q_r, k_r, v_r = _routing_inputs("small")
+    res = O.route(q_r, k_r, g, 0.0, 1, cfg.sm_scale)
+    assert (res.counts == 1).all()
+    o_r = O.sparse_attn(q_r, k_r, v_r, res.idx, res.counts, g, cfg.sm_scale)
+    bs = O.block_tokens(g)
+    qf, kf, vf = (bits_to_f64(t) for t in (q_r, k_r, v_r))
+    for h, i in [(0, 0), (3, 7), (11, 15)]:
+        j = int(res.idx[h, i, 0])
+        z = qf[h, i * bs:(i + 1) * bs] @ kf[h, j * bs:(j + 1) * bs].T * cfg.sm_scale
+        w = np.exp(z - z.max(-1, keepdims=True))
+        w /= w.sum(-1, keepdims=True)
+        np.testing.assert_allclose(o_r[h, i * bs:(i + 1) * bs], w @ vf[h, j * bs:(j + 1) * bs],
+                                   rtol=1e-10, atol=1e-12)
