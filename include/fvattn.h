@@ -1,0 +1,151 @@
+/*
+ * libfvattn — B200 (sm_100a) hot path of FVAttn's adaptive sparse attention for video DiTs:
+ *   reorder -> route (Top-p with a Top-k floor) -> block-sparse attention -> inverse reorder.
+ *
+ * C ABI.  Unless a parameter says "host", every data pointer is a DEVICE pointer owned by
+ * the caller; the library allocates no device memory and keeps no state between calls.
+ * All work is enqueued on the caller's CUDA stream (`stream` is a cudaStream_t passed as
+ * void*; NULL = the legacy default stream) and no call synchronises except
+ * fvattn_device_status.  Host-detectable problems return a status before any launch;
+ * device-detected problems (index out of range, a pipeline wait that ran out) set a sticky
+ * error word in the caller's workspace, make the kernel return cleanly, and are read back
+ * by fvattn_device_status.
+ *
+ * Notation (paper Sec. 2.1, Sec. 3.1, Eq. 1): latent grid (T,Y,X); tile = block shape
+ * (tT,tY,tX); nT = ceil(T/tT) ...; nb = nT*nY*nX blocks of Bs = tT*tY*tX tokens;
+ * N = T*Y*X tokens; N_pad = nb*Bs; H heads of dimension d; s[h,i,j] block score,
+ * M[h,i,j] block mask, L_h per-head workload.
+ *
+ * Supported shapes: d in {64,128}, Bs in {64,128}, nb <= 4096, bf16 data.
+ */
+#ifndef FVATTN_H_
+#define FVATTN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    FVATTN_OK = 0,
+    FVATTN_ERR_INVALID_ARG = 1,        /* null pointer, p NaN or > 1, k_floor < 0, misaligned pointer/stride */
+    FVATTN_ERR_UNSUPPORTED_SHAPE = 2,  /* d, Bs or nb outside the supported set */
+    FVATTN_ERR_WORKSPACE_TOO_SMALL = 3,
+    FVATTN_ERR_CUDA = 4,               /* a CUDA runtime/driver call failed (no device, launch error) */
+    FVATTN_ERR_DEVICE_TIMEOUT = 5,     /* a bounded device-side wait ran out (sticky, from the error word) */
+    FVATTN_ERR_DEVICE_BOUNDS = 6       /* an index read on the device was out of range (sticky) */
+} fvattn_status_t;
+
+/* Latent grid and tile (= block_shape). */
+typedef struct {
+    int32_t T, Y, X;
+    int32_t tT, tY, tX;
+} fvattn_grid_t;
+
+/* Caller-side token layout [B, N, H, d]: element strides, d contiguous (stride 1).
+ * Strides must be multiples of 8 elements (16-byte vectors). */
+typedef struct {
+    int32_t B, H, d;
+    int64_t stride_b, stride_n, stride_h;
+} fvattn_tok_layout_t;
+
+typedef void* fvattn_stream_t; /* cudaStream_t */
+
+/* nb, Bs, N_pad of a grid (host arithmetic only; 0 on a malformed grid). */
+int32_t fvattn_num_blocks(const fvattn_grid_t* grid);
+int32_t fvattn_block_tokens(const fvattn_grid_t* grid);
+int64_t fvattn_padded_tokens(const fvattn_grid_t* grid);
+
+/* Bytes of workspace that fvattn_route and fvattn_sparse_attn need for this shape (the
+ * larger of the two; one buffer serves both when they run back to back on one stream).
+ * The workspace must be 256-byte aligned.  Its first 256 bytes hold the sticky device
+ * error word: zero them once with fvattn_workspace_init before first use. */
+fvattn_status_t fvattn_workspace_bytes(const fvattn_grid_t* grid, int32_t B, int32_t H, int32_t d,
+                                       size_t* out_bytes /* host */);
+fvattn_status_t fvattn_workspace_init(void* workspace, size_t workspace_bytes, fvattn_stream_t stream);
+
+/*
+ * Video-aware block reorder (Sec. 3.1; 3-D tile reading).  Token (t,y,x) of `src`
+ * (layout `lay`, N in raster order over T,Y,X) goes to row blk*Bs + off of the head-major
+ * tiled tensor, blk = ((t/tT)*nY + y/tY)*nX + x/tX, off = ((t%tT)*tY + y%tY)*tX + x%tX.
+ *   src   : bf16, [B,N,H,d] by strides, 16-byte aligned.
+ *   dst_r : bf16, dense [B,H,N_pad,d], 128-byte aligned; rows that are no token's image
+ *           (padding) are written as zero.
+ */
+fvattn_status_t fvattn_reorder(const void* src, fvattn_tok_layout_t lay, const fvattn_grid_t* grid,
+                               void* dst_r, fvattn_stream_t stream);
+
+/*
+ * Inverse of fvattn_reorder: dst[n] = src_r[pi(n)], padding rows dropped (Sec. 3.1; the
+ * restoration step that closes the layer's pipeline).
+ *   src_r : bf16 [B,H,N_pad,d];  dst : bf16 [B,N,H,d] by `lay`.
+ */
+fvattn_status_t fvattn_inverse_reorder(const void* src_r, const fvattn_grid_t* grid, void* dst,
+                                       fvattn_tok_layout_t lay, fvattn_stream_t stream);
+
+/*
+ * Top-p block routing with a Top-k floor (Sec. 2.1; Sec. 3.1 pooled similarities; Eq. 1).
+ * For every head bh and query block i:
+ *   qbar, kbar = mean of the block's valid (non-padding) rows          (fp32)
+ *   s[j] = sm_scale * <qbar[i], kbar[j]>;  P = softmax_j s              (fp32)
+ *   order j by s descending, ties to the lower j
+ *   c_p = smallest m >= 1 whose first m blocks hold mass >= p  (nb if p >= 1 or never reached;
+ *         p <= 0 gives 1);   c = max(c_p, min(k_floor, nb));   keep the first c blocks.
+ * Inputs : q_r, k_r bf16 [B,H,N_pad,d] as written by fvattn_reorder.
+ * Outputs: mask_bits [B,H,nb,ceil(nb/32)] u32, bit (j&31) of word j>>5 = M[h,i,j];
+ *          counts    [B,H,nb] i32 = c;
+ *          idx       [B,H,nb,nb] u16, row (h,i): its first counts entries are the retained j
+ *                    in ascending order; the remaining entries are left untouched;
+ *          head_load [B,H] f32 = mean_i counts (Eq. 1), may be NULL.
+ * p in (-inf, 1]; k_floor >= 0.  Uses the workspace (pooled means and the score matrix).
+ */
+fvattn_status_t fvattn_route(const void* q_r, const void* k_r, int32_t B, int32_t H, int32_t d,
+                             const fvattn_grid_t* grid, float p, int32_t k_floor, float sm_scale,
+                             uint32_t* mask_bits, int32_t* counts, uint16_t* idx, float* head_load,
+                             void* workspace, size_t workspace_bytes, fvattn_stream_t stream);
+
+/*
+ * Block-sparse attention over the retained (query block, key block) pairs (Sec. 2.1): for
+ * each valid query row r of block i,
+ *   O[r] = softmax_{r' in retained blocks, r' valid}(sm_scale * <Q[r],K[r']>) . V[r'],
+ * bf16 inputs, fp32 accumulation and softmax, bf16 output; padding query rows give 0.
+ * The mask is taken in compact form (idx, counts) as written by fvattn_route; each row's
+ * entries must be distinct block indices < nb (checked on the device: a bad index sets
+ * FVATTN_ERR_DEVICE_BOUNDS and that tile is skipped).  counts[h,i] == 0 gives zero rows.
+ * (Head, query-block) tiles are handed to persistent CTAs heaviest first, head by head
+ * (heads by total retained blocks, tiles inside a head by count), built on the device from
+ * `counts` with no host round trip.
+ *   q_r,k_r,v_r : bf16 [B,H,N_pad,d], 128-byte aligned;  o_r : bf16 [B,H,N_pad,d].
+ */
+fvattn_status_t fvattn_sparse_attn(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
+                                   const int32_t* counts, int32_t B, int32_t H, int32_t d,
+                                   const fvattn_grid_t* grid, float sm_scale, void* o_r, void* workspace,
+                                   size_t workspace_bytes, fvattn_stream_t stream);
+
+/* Same contract as fvattn_sparse_attn, computed by the plain CUDA-core kernel (no tensor
+ * cores).  fvattn_sparse_attn uses it for shapes other than Bs = d = 128; exported so the
+ * two kernels can be compared on a GPU. */
+fvattn_status_t fvattn_sparse_attn_simt(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
+                                        const int32_t* counts, int32_t B, int32_t H, int32_t d,
+                                        const fvattn_grid_t* grid, float sm_scale, void* o_r, void* workspace,
+                                        size_t workspace_bytes, fvattn_stream_t stream);
+
+/* The heaviest-first tile order fvattn_sparse_attn builds from `counts` (Sec. 2.2's
+ * observation that per-head workloads differ, applied inside one GPU): order[t] = bh*nb + i.
+ * Exported for inspection and tests.  order: u32 [B*H*nb]. */
+fvattn_status_t fvattn_tile_order(const int32_t* counts, int32_t B, int32_t H, const fvattn_grid_t* grid,
+                                  uint32_t* order, void* workspace, size_t workspace_bytes,
+                                  fvattn_stream_t stream);
+
+/* Synchronises `stream`, reads the sticky error word of the workspace and returns it
+ * (FVATTN_OK, FVATTN_ERR_DEVICE_TIMEOUT, FVATTN_ERR_DEVICE_BOUNDS, or FVATTN_ERR_CUDA). */
+fvattn_status_t fvattn_device_status(const void* workspace, fvattn_stream_t stream);
+
+const char* fvattn_status_string(fvattn_status_t status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FVATTN_H_ */

@@ -1,0 +1,273 @@
+"""ctypes binding of ``libfvattn.so``: argument marshalling only.
+
+Every step of the path (reorder, routing, tile order, sparse attention, inverse reorder) runs
+in the library's CUDA kernels; PyTorch supplies device memory and the current stream.  There
+is no CPU fallback: if the library has not been built, or no CUDA device is present, the
+calls raise.
+"""
+from __future__ import annotations
+
+import ctypes
+import math
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfvattn.so")
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, ERR_DEVICE_TIMEOUT, \
+    ERR_DEVICE_BOUNDS = range(7)
+
+EXPORTS = (
+    "fvattn_num_blocks", "fvattn_block_tokens", "fvattn_padded_tokens", "fvattn_workspace_bytes",
+    "fvattn_workspace_init", "fvattn_reorder", "fvattn_inverse_reorder", "fvattn_route",
+    "fvattn_sparse_attn", "fvattn_sparse_attn_simt", "fvattn_tile_order", "fvattn_device_status",
+    "fvattn_status_string",
+)
+
+
+class FvattnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)} (status {status})")
+
+
+class _CGrid(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("T", "Y", "X", "tT", "tY", "tX")]
+
+
+class _CLayout(ctypes.Structure):
+    _fields_ = [("B", ctypes.c_int32), ("H", ctypes.c_int32), ("d", ctypes.c_int32),
+                ("stride_b", ctypes.c_int64), ("stride_n", ctypes.c_int64), ("stride_h", ctypes.c_int64)]
+
+
+@dataclass(frozen=True)
+class Grid:
+    """Latent grid (T, Y, X) and tile = block shape (tT, tY, tX)."""
+
+    T: int
+    Y: int
+    X: int
+    tT: int
+    tY: int
+    tX: int
+
+    def c(self) -> _CGrid:
+        return _CGrid(self.T, self.Y, self.X, self.tT, self.tY, self.tX)
+
+    @property
+    def tokens(self) -> int:
+        return self.T * self.Y * self.X
+
+    @property
+    def num_blocks(self) -> int:
+        return int(lib().fvattn_num_blocks(ctypes.byref(self.c())))
+
+    @property
+    def block_tokens(self) -> int:
+        return int(lib().fvattn_block_tokens(ctypes.byref(self.c())))
+
+    @property
+    def padded_tokens(self) -> int:
+        return int(lib().fvattn_padded_tokens(ctypes.byref(self.c())))
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load the C-ABI library.  Raises if it has not been built: there is no other path."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2607_16190_b200.build` "
+                "(nvcc, sm_100a).  This package has no fallback implementation.")
+        L = ctypes.CDLL(LIB_PATH)
+        L.fvattn_num_blocks.restype = ctypes.c_int32
+        L.fvattn_block_tokens.restype = ctypes.c_int32
+        L.fvattn_padded_tokens.restype = ctypes.c_int64
+        L.fvattn_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name not in ("fvattn_num_blocks", "fvattn_block_tokens", "fvattn_padded_tokens",
+                            "fvattn_status_string"):
+                getattr(L, name).restype = ctypes.c_int32
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().fvattn_status_string(ctypes.c_int32(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != OK:
+        raise FvattnError(status, where)
+
+
+def _ptr(t: torch.Tensor | None) -> ctypes.c_void_p:
+    return ctypes.c_void_p(0 if t is None else t.data_ptr())
+
+
+def _stream() -> ctypes.c_void_p:
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _need_cuda(*tensors: torch.Tensor) -> None:
+    for t in tensors:
+        if t is not None and not t.is_cuda:
+            raise ValueError("fvattn ops take CUDA tensors; there is no CPU path")
+
+
+def _layout(x: torch.Tensor) -> _CLayout:
+    B, N, H, d = x.shape
+    if x.stride(3) != 1:
+        raise ValueError("the head dimension must be contiguous")
+    return _CLayout(B, H, d, x.stride(0), x.stride(1), x.stride(2))
+
+
+# ------------------------------------------------------------------------------- workspace
+def workspace_bytes(grid: Grid, B: int, H: int, d: int) -> int:
+    out = ctypes.c_size_t(0)
+    _check(lib().fvattn_workspace_bytes(ctypes.byref(grid.c()), B, H, d, ctypes.byref(out)), "fvattn_workspace_bytes")
+    return int(out.value)
+
+
+def make_workspace(grid: Grid, B: int, H: int, d: int, device="cuda") -> torch.Tensor:
+    """Allocate (with torch) and initialise a workspace that serves route and sparse_attn."""
+    ws = torch.empty(workspace_bytes(grid, B, H, d), dtype=torch.uint8, device=device)
+    _check(lib().fvattn_workspace_init(_ptr(ws), ctypes.c_size_t(ws.numel()), _stream()), "fvattn_workspace_init")
+    return ws
+
+
+def device_status(workspace: torch.Tensor) -> int:
+    """Synchronise the current stream and return the workspace's sticky device status."""
+    return int(lib().fvattn_device_status(_ptr(workspace), _stream()))
+
+
+# ----------------------------------------------------------------------------------- ops
+def reorder(x: torch.Tensor, grid: Grid, out: torch.Tensor | None = None) -> torch.Tensor:
+    """x [B, N, H, d] bf16 (any strides with d contiguous) -> tiled [B, H, N_pad, d]."""
+    _need_cuda(x)
+    B, N, H, d = x.shape
+    assert N == grid.tokens and x.dtype == torch.bfloat16
+    if out is None:
+        out = torch.empty(B, H, grid.padded_tokens, d, dtype=torch.bfloat16, device=x.device)
+    _check(lib().fvattn_reorder(_ptr(x), _layout(x), ctypes.byref(grid.c()), _ptr(out), _stream()), "fvattn_reorder")
+    return out
+
+
+def inverse_reorder(x_r: torch.Tensor, grid: Grid, out: torch.Tensor | None = None) -> torch.Tensor:
+    """tiled [B, H, N_pad, d] -> [B, N, H, d] (padding rows dropped)."""
+    _need_cuda(x_r)
+    B, H, n_pad, d = x_r.shape
+    assert n_pad == grid.padded_tokens and x_r.is_contiguous() and x_r.dtype == torch.bfloat16
+    if out is None:
+        out = torch.empty(B, grid.tokens, H, d, dtype=torch.bfloat16, device=x_r.device)
+    _check(lib().fvattn_inverse_reorder(_ptr(x_r), ctypes.byref(grid.c()), _ptr(out), _layout(out), _stream()),
+           "fvattn_inverse_reorder")
+    return out
+
+
+@dataclass
+class Routing:
+    mask_bits: torch.Tensor   # [B, H, nb, ceil(nb/32)] uint32
+    counts: torch.Tensor      # [B, H, nb] int32
+    idx: torch.Tensor         # [B, H, nb, nb] uint16; first counts entries valid, ascending
+    head_load: torch.Tensor   # [B, H] float32 (Eq. 1)
+
+
+def alloc_routing(grid: Grid, B: int, H: int, device="cuda") -> Routing:
+    nb = grid.num_blocks
+    return Routing(
+        mask_bits=torch.empty(B, H, nb, (nb + 31) // 32, dtype=torch.uint32, device=device),
+        counts=torch.empty(B, H, nb, dtype=torch.int32, device=device),
+        idx=torch.empty(B, H, nb, nb, dtype=torch.uint16, device=device),
+        head_load=torch.empty(B, H, dtype=torch.float32, device=device),
+    )
+
+
+def route(q_r: torch.Tensor, k_r: torch.Tensor, grid: Grid, p: float, k_floor: int, sm_scale: float | None,
+          workspace: torch.Tensor, out: Routing | None = None) -> Routing:
+    """Top-p block routing with a Top-k floor on tiled q_r, k_r [B, H, N_pad, d]."""
+    _need_cuda(q_r, k_r, workspace)
+    B, H, n_pad, d = q_r.shape
+    assert k_r.shape == q_r.shape and q_r.is_contiguous() and k_r.is_contiguous()
+    if sm_scale is None:
+        sm_scale = 1.0 / math.sqrt(d)
+    if out is None:
+        out = alloc_routing(grid, B, H, q_r.device)
+    _check(lib().fvattn_route(_ptr(q_r), _ptr(k_r), B, H, d, ctypes.byref(grid.c()), ctypes.c_float(p),
+                              ctypes.c_int32(k_floor), ctypes.c_float(sm_scale), _ptr(out.mask_bits),
+                              _ptr(out.counts), _ptr(out.idx), _ptr(out.head_load), _ptr(workspace),
+                              ctypes.c_size_t(workspace.numel()), _stream()), "fvattn_route")
+    return out
+
+
+def _attn(fn_name: str, q_r, k_r, v_r, idx, counts, grid, sm_scale, workspace, out):
+    _need_cuda(q_r, k_r, v_r, idx, counts, workspace)
+    B, H, n_pad, d = q_r.shape
+    assert all(t.is_contiguous() for t in (q_r, k_r, v_r, idx, counts))
+    assert idx.dtype == torch.uint16 and counts.dtype == torch.int32
+    if sm_scale is None:
+        sm_scale = 1.0 / math.sqrt(d)
+    if out is None:
+        out = torch.empty_like(q_r)
+    _check(getattr(lib(), fn_name)(_ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(idx), _ptr(counts), B, H, d,
+                                   ctypes.byref(grid.c()), ctypes.c_float(sm_scale), _ptr(out), _ptr(workspace),
+                                   ctypes.c_size_t(workspace.numel()), _stream()), fn_name)
+    return out
+
+
+def sparse_attn(q_r, k_r, v_r, idx, counts, grid: Grid, sm_scale: float | None, workspace: torch.Tensor,
+                out: torch.Tensor | None = None) -> torch.Tensor:
+    """Block-sparse attention over the retained pairs (idx, counts) -> o_r [B, H, N_pad, d]."""
+    return _attn("fvattn_sparse_attn", q_r, k_r, v_r, idx, counts, grid, sm_scale, workspace, out)
+
+
+def sparse_attn_simt(q_r, k_r, v_r, idx, counts, grid: Grid, sm_scale: float | None, workspace: torch.Tensor,
+                     out: torch.Tensor | None = None) -> torch.Tensor:
+    """Same contract on the CUDA-core kernel (cross-check; the path for Bs or d = 64)."""
+    return _attn("fvattn_sparse_attn_simt", q_r, k_r, v_r, idx, counts, grid, sm_scale, workspace, out)
+
+
+def tile_order(counts: torch.Tensor, grid: Grid, workspace: torch.Tensor) -> torch.Tensor:
+    """Heaviest-first order of the (head, query-block) tiles: uint32 [B*H*nb], entries bh*nb+i."""
+    _need_cuda(counts, workspace)
+    B, H, nb = counts.shape
+    order = torch.empty(B * H * nb, dtype=torch.uint32, device=counts.device)
+    _check(lib().fvattn_tile_order(_ptr(counts), B, H, ctypes.byref(grid.c()), _ptr(order), _ptr(workspace),
+                                   ctypes.c_size_t(workspace.numel()), _stream()), "fvattn_tile_order")
+    return order
+
+
+# ------------------------------------------------------------------------------ whole layer
+class SparseAttentionLayer:
+    """One attention layer of the path with every buffer preallocated (no allocation per call):
+    reorder Q,K,V -> route -> block-sparse attention -> inverse reorder."""
+
+    def __init__(self, grid: Grid, B: int, H: int, d: int, p: float, k_floor: int, sm_scale: float | None = None,
+                 device="cuda"):
+        self.grid, self.B, self.H, self.d = grid, B, H, d
+        self.p, self.k_floor = p, k_floor
+        self.sm_scale = sm_scale if sm_scale is not None else 1.0 / math.sqrt(d)
+        n_pad = grid.padded_tokens
+        self.q_r = torch.empty(B, H, n_pad, d, dtype=torch.bfloat16, device=device)
+        self.k_r = torch.empty_like(self.q_r)
+        self.v_r = torch.empty_like(self.q_r)
+        self.o_r = torch.empty_like(self.q_r)
+        self.out = torch.empty(B, grid.tokens, H, d, dtype=torch.bfloat16, device=device)
+        self.routing = alloc_routing(grid, B, H, device)
+        self.workspace = make_workspace(grid, B, H, d, device)
+
+    def __call__(self, q: torch.Tensor, k: torch.Tensor, v: torch.Tensor) -> torch.Tensor:
+        g = self.grid
+        reorder(q, g, self.q_r)
+        reorder(k, g, self.k_r)
+        reorder(v, g, self.v_r)
+        route(self.q_r, self.k_r, g, self.p, self.k_floor, self.sm_scale, self.workspace, self.routing)
+        sparse_attn(self.q_r, self.k_r, self.v_r, self.routing.idx, self.routing.counts, g, self.sm_scale,
+                    self.workspace, self.o_r)
+        return inverse_reorder(self.o_r, g, self.out)

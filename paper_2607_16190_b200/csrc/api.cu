@@ -1,0 +1,170 @@
+// extern "C" entry points of libfvattn: argument validation and dispatch.  Nothing here
+// allocates device memory or synchronises (except fvattn_device_status).
+#include <math.h>
+
+#include "common.cuh"
+
+using namespace fvattn;
+
+namespace {
+
+bool shape_ok(int d, const GridDims& m) {
+    return (d == 64 || d == 128) && (m.bs == 64 || m.bs == 128) && m.nb >= 1 && m.nb <= kMaxBlocks;
+}
+
+fvattn_status_t check_layout(const fvattn_tok_layout_t& lay, const void* tok, const void* tiled,
+                             const fvattn_grid_t* grid) {
+    if (!tok || !tiled || !grid_ok(grid)) return FVATTN_ERR_INVALID_ARG;
+    if (lay.B <= 0 || lay.H <= 0 || lay.d <= 0) return FVATTN_ERR_INVALID_ARG;
+    if (lay.d % 8 != 0) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if (lay.stride_b % 8 || lay.stride_n % 8 || lay.stride_h % 8) return FVATTN_ERR_INVALID_ARG;
+    if (lay.stride_n < lay.d || lay.stride_h < lay.d || lay.stride_b < 0) return FVATTN_ERR_INVALID_ARG;
+    if (!aligned(tok, 16) || !aligned(tiled, 16)) return FVATTN_ERR_INVALID_ARG;
+    if ((int64_t)lay.B * lay.H > 65535 * 8 || lay.B > 65535) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    return FVATTN_OK;
+}
+
+fvattn_status_t check_attn_args(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
+                                const int32_t* counts, int32_t B, int32_t H, int32_t d, const fvattn_grid_t* grid,
+                                float sm_scale, void* o_r, void* workspace, size_t workspace_bytes) {
+    if (!q_r || !k_r || !v_r || !idx || !counts || !o_r || !workspace || !grid_ok(grid))
+        return FVATTN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || !(sm_scale == sm_scale) || isinf(sm_scale)) return FVATTN_ERR_INVALID_ARG;
+    GridDims m = make_dims(*grid);
+    if (!shape_ok(d, m)) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if ((int64_t)B * H * m.nb > 0x7fffffffLL) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(q_r, 128) || !aligned(k_r, 128) || !aligned(v_r, 128) || !aligned(o_r, 128) ||
+        !aligned(workspace, 256) || !aligned(idx, 2) || !aligned(counts, 4))
+        return FVATTN_ERR_INVALID_ARG;
+    if (workspace_bytes < attn_ws((int64_t)B * H, m.nb).total) return FVATTN_ERR_WORKSPACE_TOO_SMALL;
+    return FVATTN_OK;
+}
+
+} // namespace
+
+extern "C" {
+
+int32_t fvattn_num_blocks(const fvattn_grid_t* grid) { return grid_ok(grid) ? make_dims(*grid).nb : 0; }
+int32_t fvattn_block_tokens(const fvattn_grid_t* grid) { return grid_ok(grid) ? make_dims(*grid).bs : 0; }
+int64_t fvattn_padded_tokens(const fvattn_grid_t* grid) { return grid_ok(grid) ? make_dims(*grid).n_pad : 0; }
+
+fvattn_status_t fvattn_workspace_bytes(const fvattn_grid_t* grid, int32_t B, int32_t H, int32_t d,
+                                       size_t* out_bytes) {
+    if (!out_bytes || !grid_ok(grid) || B <= 0 || H <= 0) return FVATTN_ERR_INVALID_ARG;
+    GridDims m = make_dims(*grid);
+    if (!shape_ok(d, m)) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    size_t a = route_ws((int64_t)B * H, m.nb, d).total, b = attn_ws((int64_t)B * H, m.nb).total;
+    *out_bytes = a > b ? a : b;
+    return FVATTN_OK;
+}
+
+fvattn_status_t fvattn_workspace_init(void* workspace, size_t workspace_bytes, fvattn_stream_t stream) {
+    if (!workspace || workspace_bytes < kWsHeaderBytes || !aligned(workspace, 256)) return FVATTN_ERR_INVALID_ARG;
+    FVATTN_CUDA_OK(cudaMemsetAsync(workspace, 0, kWsHeaderBytes, (cudaStream_t)stream));
+    return FVATTN_OK;
+}
+
+fvattn_status_t fvattn_reorder(const void* src, fvattn_tok_layout_t lay, const fvattn_grid_t* grid, void* dst_r,
+                               fvattn_stream_t stream) {
+    fvattn_status_t st = check_layout(lay, src, dst_r, grid);
+    if (st != FVATTN_OK) return st;
+    return launch_reorder(src, lay, make_dims(*grid), dst_r, (cudaStream_t)stream);
+}
+
+fvattn_status_t fvattn_inverse_reorder(const void* src_r, const fvattn_grid_t* grid, void* dst,
+                                       fvattn_tok_layout_t lay, fvattn_stream_t stream) {
+    fvattn_status_t st = check_layout(lay, dst, src_r, grid);
+    if (st != FVATTN_OK) return st;
+    return launch_inverse_reorder(src_r, make_dims(*grid), dst, lay, (cudaStream_t)stream);
+}
+
+fvattn_status_t fvattn_route(const void* q_r, const void* k_r, int32_t B, int32_t H, int32_t d,
+                             const fvattn_grid_t* grid, float p, int32_t k_floor, float sm_scale,
+                             uint32_t* mask_bits, int32_t* counts, uint16_t* idx, float* head_load, void* workspace,
+                             size_t workspace_bytes, fvattn_stream_t stream) {
+    if (!q_r || !k_r || !mask_bits || !counts || !idx || !workspace || !grid_ok(grid)) return FVATTN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || k_floor < 0) return FVATTN_ERR_INVALID_ARG;
+    if (!(p == p) || p > 1.0f || !(sm_scale == sm_scale) || isinf(sm_scale)) return FVATTN_ERR_INVALID_ARG;
+    GridDims m = make_dims(*grid);
+    if (!shape_ok(d, m)) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if ((int64_t)B * H > 65535) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(q_r, 16) || !aligned(k_r, 16) || !aligned(workspace, 256) || !aligned(mask_bits, 4) ||
+        !aligned(counts, 4) || !aligned(idx, 2) || (head_load && !aligned(head_load, 4)))
+        return FVATTN_ERR_INVALID_ARG;
+    if (workspace_bytes < route_ws((int64_t)B * H, m.nb, d).total) return FVATTN_ERR_WORKSPACE_TOO_SMALL;
+    return launch_route(q_r, k_r, (int64_t)B * H, d, m, p, k_floor, sm_scale, mask_bits, counts, idx, head_load,
+                        workspace, (cudaStream_t)stream);
+}
+
+fvattn_status_t fvattn_tile_order(const int32_t* counts, int32_t B, int32_t H, const fvattn_grid_t* grid,
+                                  uint32_t* order, void* workspace, size_t workspace_bytes, fvattn_stream_t stream) {
+    if (!counts || !order || !workspace || !grid_ok(grid) || B <= 0 || H <= 0) return FVATTN_ERR_INVALID_ARG;
+    GridDims m = make_dims(*grid);
+    if (m.nb > kMaxBlocks || (int64_t)B * H * m.nb > 0x7fffffffLL) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(workspace, 256) || !aligned(order, 4) || !aligned(counts, 4)) return FVATTN_ERR_INVALID_ARG;
+    if (workspace_bytes < attn_ws((int64_t)B * H, m.nb).total) return FVATTN_ERR_WORKSPACE_TOO_SMALL;
+    return launch_tile_order(counts, (int64_t)B * H, m.nb, order, workspace, (cudaStream_t)stream);
+}
+
+fvattn_status_t fvattn_sparse_attn_simt(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
+                                        const int32_t* counts, int32_t B, int32_t H, int32_t d,
+                                        const fvattn_grid_t* grid, float sm_scale, void* o_r, void* workspace,
+                                        size_t workspace_bytes, fvattn_stream_t stream) {
+    fvattn_status_t st = check_attn_args(q_r, k_r, v_r, idx, counts, B, H, d, grid, sm_scale, o_r, workspace,
+                                         workspace_bytes);
+    if (st != FVATTN_OK) return st;
+    GridDims m = make_dims(*grid);
+    const int64_t BH = (int64_t)B * H;
+    uint32_t* order = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + attn_ws(BH, m.nb).order);
+    st = launch_tile_order(counts, BH, m.nb, order, workspace, (cudaStream_t)stream);
+    if (st != FVATTN_OK) return st;
+    return launch_attn_simt(q_r, k_r, v_r, idx, counts, BH, d, m, sm_scale, o_r, order, workspace,
+                            (cudaStream_t)stream);
+}
+
+fvattn_status_t fvattn_sparse_attn(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
+                                   const int32_t* counts, int32_t B, int32_t H, int32_t d, const fvattn_grid_t* grid,
+                                   float sm_scale, void* o_r, void* workspace, size_t workspace_bytes,
+                                   fvattn_stream_t stream) {
+    fvattn_status_t st = check_attn_args(q_r, k_r, v_r, idx, counts, B, H, d, grid, sm_scale, o_r, workspace,
+                                         workspace_bytes);
+    if (st != FVATTN_OK) return st;
+    GridDims m = make_dims(*grid);
+    const int64_t BH = (int64_t)B * H;
+    uint32_t* order = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + attn_ws(BH, m.nb).order);
+    st = launch_tile_order(counts, BH, m.nb, order, workspace, (cudaStream_t)stream);
+    if (st != FVATTN_OK) return st;
+    if (m.bs == 128 && d == 128)
+        return launch_attn_tc(q_r, k_r, v_r, idx, counts, BH, m, sm_scale, o_r, order, workspace,
+                              (cudaStream_t)stream);
+    return launch_attn_simt(q_r, k_r, v_r, idx, counts, BH, d, m, sm_scale, o_r, order, workspace,
+                            (cudaStream_t)stream);
+}
+
+fvattn_status_t fvattn_device_status(const void* workspace, fvattn_stream_t stream) {
+    if (!workspace) return FVATTN_ERR_INVALID_ARG;
+    WsHeader h;
+    FVATTN_CUDA_OK(cudaMemcpyAsync(&h, workspace, sizeof(h), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    FVATTN_CUDA_OK(cudaStreamSynchronize((cudaStream_t)stream));
+    switch (h.status) {
+        case 0: return FVATTN_OK;
+        case FVATTN_ERR_DEVICE_TIMEOUT: return FVATTN_ERR_DEVICE_TIMEOUT;
+        case FVATTN_ERR_DEVICE_BOUNDS: return FVATTN_ERR_DEVICE_BOUNDS;
+        default: return FVATTN_ERR_CUDA;
+    }
+}
+
+const char* fvattn_status_string(fvattn_status_t status) {
+    switch (status) {
+        case FVATTN_OK: return "ok";
+        case FVATTN_ERR_INVALID_ARG: return "invalid argument";
+        case FVATTN_ERR_UNSUPPORTED_SHAPE: return "unsupported shape";
+        case FVATTN_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case FVATTN_ERR_CUDA: return "CUDA error";
+        case FVATTN_ERR_DEVICE_TIMEOUT: return "device-side wait timed out";
+        case FVATTN_ERR_DEVICE_BOUNDS: return "device-side index out of range";
+    }
+    return "unknown status";
+}
+
+} // extern "C"

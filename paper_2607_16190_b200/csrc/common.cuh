@@ -1,0 +1,149 @@
+// Shared declarations of the library's translation units: grid arithmetic, workspace layout,
+// the sticky device error word, launch helpers.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "fvattn.h"
+
+namespace fvattn {
+
+// ---- grid arithmetic (Sec. 3.1, tile reading) ------------------------------------------
+struct GridDims {
+    int T, Y, X, tT, tY, tX;
+    int nT, nY, nX;
+    int nb;        // blocks
+    int bs;        // tokens per block
+    int64_t n;     // tokens
+    int64_t n_pad; // nb * bs
+};
+
+__host__ __device__ inline GridDims make_dims(const fvattn_grid_t& g) {
+    GridDims m;
+    m.T = g.T; m.Y = g.Y; m.X = g.X; m.tT = g.tT; m.tY = g.tY; m.tX = g.tX;
+    m.nT = (g.T + g.tT - 1) / g.tT;
+    m.nY = (g.Y + g.tY - 1) / g.tY;
+    m.nX = (g.X + g.tX - 1) / g.tX;
+    m.nb = m.nT * m.nY * m.nX;
+    m.bs = g.tT * g.tY * g.tX;
+    m.n = (int64_t)g.T * g.Y * g.X;
+    m.n_pad = (int64_t)m.nb * m.bs;
+    return m;
+}
+
+inline bool grid_ok(const fvattn_grid_t* g) {
+    if (!g) return false;
+    if (g->T <= 0 || g->Y <= 0 || g->X <= 0 || g->tT <= 0 || g->tY <= 0 || g->tX <= 0) return false;
+    if ((int64_t)g->tT * g->tY * g->tX > 65536) return false;
+    int64_t nb = (int64_t)((g->T + g->tT - 1) / g->tT) * ((g->Y + g->tY - 1) / g->tY) * ((g->X + g->tX - 1) / g->tX);
+    return nb <= (1 << 24);
+}
+
+// Coordinates of row `off` of block `blk`; returns whether the row is a token (not padding).
+__device__ __forceinline__ bool row_to_token(const GridDims& m, int blk, int off, int64_t* token) {
+    int bx = blk % m.nX;
+    int by = (blk / m.nX) % m.nY;
+    int bt = blk / (m.nX * m.nY);
+    int ox = off % m.tX;
+    int oy = (off / m.tX) % m.tY;
+    int ot = off / (m.tX * m.tY);
+    int t = bt * m.tT + ot, y = by * m.tY + oy, x = bx * m.tX + ox;
+    *token = ((int64_t)t * m.Y + y) * m.X + x;
+    return t < m.T && y < m.Y && x < m.X;
+}
+
+// Number of valid tokens of a block (closed form).
+__host__ __device__ inline int block_valid_tokens(const GridDims& m, int blk) {
+    int bx = blk % m.nX;
+    int by = (blk / m.nX) % m.nY;
+    int bt = blk / (m.nX * m.nY);
+    int vt = min(m.tT, m.T - bt * m.tT);
+    int vy = min(m.tY, m.Y - by * m.tY);
+    int vx = min(m.tX, m.X - bx * m.tX);
+    return vt * vy * vx;
+}
+
+// ---- workspace ------------------------------------------------------------------------
+// [0, 256): header.  word 0 = sticky status, word 1 = detail, word 2 = tile counter of the
+// persistent attention kernel, word 3 = CTAs that finished (used to re-arm the counter).
+constexpr size_t kWsHeaderBytes = 256;
+constexpr int kMaxBlocks = 4096;
+
+struct WsHeader {
+    unsigned int status;
+    unsigned int detail;
+    unsigned int tile_counter;
+    unsigned int reserved;
+};
+
+__device__ __forceinline__ void report_error(void* workspace, unsigned int status, unsigned int detail) {
+    WsHeader* h = reinterpret_cast<WsHeader*>(workspace);
+    if (atomicCAS(&h->status, 0u, status) == 0u) h->detail = detail;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+struct RouteWs {
+    size_t qbar, kbar, scores, total;
+    int score_stride; // floats per score row
+};
+inline RouteWs route_ws(int64_t BH, int nb, int d) {
+    RouteWs w;
+    w.score_stride = (nb + 3) / 4 * 4;
+    size_t off = kWsHeaderBytes;
+    w.qbar = off; off = align_up(off + sizeof(float) * (size_t)BH * nb * d, 256);
+    w.kbar = off; off = align_up(off + sizeof(float) * (size_t)BH * nb * d, 256);
+    w.scores = off; off = align_up(off + sizeof(float) * (size_t)BH * nb * w.score_stride, 256);
+    w.total = off;
+    return w;
+}
+
+struct AttnWs {
+    size_t head_sum, order, total;
+};
+inline AttnWs attn_ws(int64_t BH, int nb) {
+    AttnWs w;
+    size_t off = kWsHeaderBytes;
+    w.head_sum = off; off = align_up(off + sizeof(unsigned int) * (size_t)BH, 256);
+    w.order = off; off = align_up(off + sizeof(unsigned int) * (size_t)BH * nb, 256);
+    w.total = off;
+    return w;
+}
+
+// ---- host helpers -----------------------------------------------------------------------
+#define FVATTN_CUDA_OK(expr)                         \
+    do {                                             \
+        cudaError_t e__ = (expr);                    \
+        if (e__ != cudaSuccess) {                    \
+            (void)cudaGetLastError();                \
+            return FVATTN_ERR_CUDA;                  \
+        }                                            \
+    } while (0)
+
+inline fvattn_status_t launch_status() {
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? FVATTN_OK : FVATTN_ERR_CUDA;
+}
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// ---- kernel launchers implemented by the other translation units -------------------------
+fvattn_status_t launch_reorder(const void* src, const fvattn_tok_layout_t& lay, const GridDims& m, void* dst_r,
+                               cudaStream_t s);
+fvattn_status_t launch_inverse_reorder(const void* src_r, const GridDims& m, void* dst,
+                                       const fvattn_tok_layout_t& lay, cudaStream_t s);
+fvattn_status_t launch_route(const void* q_r, const void* k_r, int64_t BH, int d, const GridDims& m, float p,
+                             int k_floor, float sm_scale, uint32_t* mask_bits, int32_t* counts, uint16_t* idx,
+                             float* head_load, void* workspace, cudaStream_t s);
+fvattn_status_t launch_tile_order(const int32_t* counts, int64_t BH, int nb, uint32_t* order, void* workspace,
+                                  cudaStream_t s);
+fvattn_status_t launch_attn_simt(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
+                                 const int32_t* counts, int64_t BH, int d, const GridDims& m, float sm_scale,
+                                 void* o_r, const uint32_t* order, void* workspace, cudaStream_t s);
+fvattn_status_t launch_attn_tc(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
+                               const int32_t* counts, int64_t BH, const GridDims& m, float sm_scale, void* o_r,
+                               const uint32_t* order, void* workspace, cudaStream_t s);
+
+} // namespace fvattn

@@ -1,0 +1,104 @@
+// Intra-GPU tile scheduler order.  The paper balances heterogeneous per-head workloads
+// (Eq. 1, Sec. 2.2) across GPUs; on one GPU the same imbalance shows up as persistent CTAs
+// idling behind a few heavy (head, query-block) tiles.  The order built here hands tiles out
+// heaviest first in two levels: heads by total retained blocks (descending), tiles inside a
+// head by their retained-block count (descending).  Keeping one head's tiles adjacent keeps
+// that head's K/V resident in L2 while its tiles are in flight.  Built on the device from
+// `counts`: no host round trip.
+#include "common.cuh"
+
+namespace fvattn {
+
+__global__ void __launch_bounds__(256)
+head_sum_kernel(const int32_t* __restrict__ counts, int nb, unsigned int* __restrict__ head_sum, WsHeader* hdr) {
+    __shared__ unsigned int red[8];
+    const int64_t bh = blockIdx.x;
+    unsigned int s = 0;
+    for (int i = threadIdx.x; i < nb; i += 256) s += (unsigned int)min(max(counts[bh * nb + i], 0), nb);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned int t = 0;
+        for (int w = 0; w < 8; ++w) t += red[w];
+        head_sum[bh] = t;
+        if (bh == 0 && hdr) hdr->tile_counter = 0u;   // re-arm the persistent kernel's queue
+    }
+}
+
+// dynamic smem: hist u32[nb + 1]
+__global__ void __launch_bounds__(256)
+tile_order_kernel(const int32_t* __restrict__ counts, int nb, int BH, const unsigned int* __restrict__ head_sum,
+                  uint32_t* __restrict__ order) {
+    extern __shared__ unsigned int hist[];
+    __shared__ unsigned int chunk_tot[256];
+    __shared__ int rank_s;
+    const int bh = blockIdx.x;
+    const int tid = threadIdx.x;
+    const int bins = nb + 1;
+
+    if (tid == 0) rank_s = 0;
+    for (int c = tid; c < bins; c += 256) hist[c] = 0u;
+    __syncthreads();
+
+    // rank of this head: heads with a larger sum (or equal sum and lower index) come first
+    const unsigned int mine = head_sum[bh];
+    int ahead = 0;
+    for (int h = tid; h < BH; h += 256) {
+        unsigned int o = head_sum[h];
+        ahead += (o > mine) || (o == mine && h < bh);
+    }
+    if (ahead) atomicAdd(&rank_s, ahead);
+    for (int i = tid; i < nb; i += 256) atomicAdd(&hist[min(max(counts[(int64_t)bh * nb + i], 0), nb)], 1u);
+    __syncthreads();
+
+    // start[c] = number of tiles with a larger count: suffix sums over the bins, in chunks
+    const int chunk = (bins + 255) / 256;
+    const int hi = bins - 1 - tid * chunk;          // this thread owns bins hi, hi-1, ..., hi-chunk+1
+    unsigned int tot = 0;
+    for (int e = 0; e < chunk; ++e) {
+        int c = hi - e;
+        if (c >= 0) tot += hist[c];
+    }
+    chunk_tot[tid] = tot;
+    __syncthreads();
+    if (tid == 0) {
+        unsigned int run = 0;
+        for (int t = 0; t < 256; ++t) {
+            unsigned int v = chunk_tot[t];
+            chunk_tot[t] = run;
+            run += v;
+        }
+    }
+    __syncthreads();
+    unsigned int run = chunk_tot[tid];
+    for (int e = 0; e < chunk; ++e) {
+        int c = hi - e;
+        if (c >= 0) {
+            unsigned int v = hist[c];
+            hist[c] = run;     // becomes the next free slot of bin c
+            run += v;
+        }
+    }
+    __syncthreads();
+    uint32_t* out = order + (int64_t)rank_s * nb;
+    for (int i = tid; i < nb; i += 256) {
+        int c = min(max(counts[(int64_t)bh * nb + i], 0), nb);
+        unsigned int pos = atomicAdd(&hist[c], 1u);
+        out[pos] = (uint32_t)((int64_t)bh * nb + i);
+    }
+}
+
+fvattn_status_t launch_tile_order(const int32_t* counts, int64_t BH, int nb, uint32_t* order, void* workspace,
+                                  cudaStream_t s) {
+    WsHeader* hdr = reinterpret_cast<WsHeader*>(workspace);
+    unsigned int* head_sum = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + attn_ws(BH, nb).head_sum);
+    head_sum_kernel<<<(unsigned)BH, 256, 0, s>>>(counts, nb, head_sum, hdr);
+    if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
+    tile_order_kernel<<<(unsigned)BH, 256, sizeof(unsigned int) * (size_t)(nb + 1), s>>>(counts, nb, (int)BH,
+                                                                                      head_sum, order);
+    return launch_status();
+}
+
+} // namespace fvattn

@@ -1,0 +1,93 @@
+"""CPU-side checks of the C-ABI library: it loads, exports every symbol the header declares,
+its host arithmetic matches the closed forms, and host-detectable errors are returned before
+any launch.  No compute call needs a GPU here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2607_16190_b200 import binding as fv
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "fvattn.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(fvattn_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    L = fv.lib()
+    names = declared_symbols()
+    assert len(names) >= 12
+    for n in names:
+        assert hasattr(L, n), n
+    assert set(names) == set(fv.EXPORTS)
+
+
+def test_grid_arithmetic_closed_forms():
+    g = fv.Grid(21, 45, 80, 1, 8, 16)
+    assert (g.num_blocks, g.block_tokens, g.padded_tokens) == (630, 128, 80640)
+    g = fv.Grid(21, 30, 52, 1, 8, 16)
+    assert (g.num_blocks, g.block_tokens, g.padded_tokens) == (336, 128, 43008)
+    g = fv.Grid(4, 8, 8, 1, 8, 8)
+    assert (g.num_blocks, g.block_tokens, g.padded_tokens) == (4, 64, 256)
+    assert fv.Grid(0, 8, 8, 1, 8, 8).num_blocks == 0          # malformed grid
+
+
+def test_workspace_bytes_and_shape_errors():
+    g = fv.Grid(21, 45, 80, 1, 8, 16)
+    n = fv.workspace_bytes(g, 1, 40, 128)
+    nb = 630
+    # header + two pooled-mean tensors + the score matrix (row stride rounded to 4 floats)
+    assert n >= 256 + 2 * 40 * nb * 128 * 4 + 40 * nb * 632 * 4
+    assert n < 256 + 2 * 40 * nb * 128 * 4 + 40 * nb * 632 * 4 + 4096
+    with pytest.raises(fv.FvattnError) as e:
+        fv.workspace_bytes(g, 1, 40, 96)                      # d not in {64, 128}
+    assert e.value.status == fv.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(fv.FvattnError) as e:
+        fv.workspace_bytes(fv.Grid(4, 8, 8, 1, 4, 8), 1, 2, 64)   # Bs = 32
+    assert e.value.status == fv.ERR_UNSUPPORTED_SHAPE
+    with pytest.raises(fv.FvattnError) as e:
+        fv.workspace_bytes(fv.Grid(64, 128, 128, 1, 8, 16), 1, 2, 128)   # nb = 8192 > 4096
+    assert e.value.status == fv.ERR_UNSUPPORTED_SHAPE
+
+
+def test_null_and_bad_arguments_are_rejected_on_the_host():
+    L = fv.lib()
+    g = fv.Grid(4, 8, 8, 1, 8, 8).c()
+    null = ctypes.c_void_p(0)
+    fake = ctypes.c_void_p(0x10000)      # never dereferenced: validation fails first
+    st = L.fvattn_route(null, fake, 1, 2, 64, ctypes.byref(g), ctypes.c_float(0.9), 1, ctypes.c_float(0.125),
+                        fake, fake, fake, null, fake, ctypes.c_size_t(1 << 20), null)
+    assert st == fv.ERR_INVALID_ARG
+    st = L.fvattn_route(fake, fake, 1, 2, 64, ctypes.byref(g), ctypes.c_float(1.5), 1, ctypes.c_float(0.125),
+                        fake, fake, fake, null, fake, ctypes.c_size_t(1 << 20), null)
+    assert st == fv.ERR_INVALID_ARG      # p > 1
+    st = L.fvattn_route(fake, fake, 1, 2, 64, ctypes.byref(g), ctypes.c_float(float("nan")), 1,
+                        ctypes.c_float(0.125), fake, fake, fake, null, fake, ctypes.c_size_t(1 << 20), null)
+    assert st == fv.ERR_INVALID_ARG      # p NaN
+    st = L.fvattn_route(fake, fake, 1, 2, 64, ctypes.byref(g), ctypes.c_float(0.9), -1, ctypes.c_float(0.125),
+                        fake, fake, fake, null, fake, ctypes.c_size_t(1 << 20), null)
+    assert st == fv.ERR_INVALID_ARG      # k_floor < 0
+    st = L.fvattn_route(fake, fake, 1, 2, 64, ctypes.byref(g), ctypes.c_float(0.9), 1, ctypes.c_float(0.125),
+                        fake, fake, fake, null, fake, ctypes.c_size_t(512), null)
+    assert st == fv.ERR_WORKSPACE_TOO_SMALL
+    st = L.fvattn_sparse_attn(fake, fake, fake, fake, fake, 1, 2, 64, ctypes.byref(g), ctypes.c_float(0.125),
+                              fake, fake, ctypes.c_size_t(16), null)
+    assert st == fv.ERR_WORKSPACE_TOO_SMALL
+    st = L.fvattn_sparse_attn(fake, fake, ctypes.c_void_p(0x10008), fake, fake, 1, 2, 64, ctypes.byref(g),
+                              ctypes.c_float(0.125), fake, fake, ctypes.c_size_t(1 << 20), null)
+    assert st == fv.ERR_INVALID_ARG      # v_r not 128-byte aligned
+    assert fv.status_string(fv.ERR_DEVICE_TIMEOUT) == "device-side wait timed out"
+
+
+def test_ops_refuse_cpu_tensors():
+    import torch
+
+    g = fv.Grid(4, 8, 8, 1, 8, 8)
+    x = torch.zeros(1, 256, 2, 64, dtype=torch.bfloat16)
+    with pytest.raises(ValueError):
+        fv.reorder(x, g)
