@@ -1,0 +1,397 @@
+#!/usr/bin/env python
+"""Benchmark of the FVAttn hot path on B200.
+
+One "step" = one attention layer of the path on one batch of synthetic Wan2.2-shaped inputs:
+reorder(Q, K, V) -> route (Top-p, Top-k floor) -> block-sparse attention -> inverse reorder.
+Prints ONE JSON line (rank 0).  `value` is effective TFLOP/s over the whole step
+(4*d*Bq*Bk FLOP per retained block pair / step time) with inputs resident in HBM; `e2e` is the
+same metric with pinned HOST inputs copied in and the output copied back inside the timed
+region; `roofline` describes the dominant kernel (the sparse attention kernel); `cpu_baseline`
+is the fp64 CPU oracle timed on this machine's host cores on a bounded sample.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload wan720p] [--impl reference]
+  torchrun ... bench.py --gpus N ...      (N independent replicas, one per GPU: the path does
+                                           not shard across GPUs; value = N x units / max time)
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FLOP_PER_PAIR = 4 * 128 * 128 * 128          # 4*d*Bq*Bk, d = Bq = Bk = 128
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+METRIC = "sparse-attn effective TFLOPS per attention layer (4*d*Bq*Bk FLOP per retained block pair / time)"
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_tc_kernel launch, from the ncu capture
+# summarised under profiles/; None until a capture of the current kernel exists.
+ATTN_DRAM_TRAFFIC_BYTES_PER_PAIR = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.samples = []
+        self._stop = threading.Event()
+        self._thread = threading.Thread(target=self._run, daemon=True)
+
+    def _run(self):
+        while not self._stop.is_set():
+            try:
+                out = subprocess.run(["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.QUERY}",
+                                      "--format=csv,noheader,nounits"], capture_output=True, text=True, timeout=5)
+                parts = [p.strip() for p in out.stdout.strip().split(",")]
+                if len(parts) == 6:
+                    self.samples.append(parts)
+            except Exception:
+                pass
+            self._stop.wait(0.2)
+
+    def __enter__(self):
+        self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        self._thread.join(timeout=10)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = sorted(float(s[0]) for s in self.samples)
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for k, n in enumerate(names) if any(s[2 + k].lower().startswith("active") for s in self.samples)]
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": float(self.samples[0][1]), "reasons": reasons,
+                "samples": len(sm)}
+
+
+def dist_env():
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    return rank, world, local
+
+
+def time_steps(fn, steps, torch):
+    """CUDA-event time of `steps` calls of fn on the current stream, in ms (total)."""
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    a.record()
+    for _ in range(steps):
+        fn()
+    b.record()
+    torch.cuda.synchronize()
+    return a.elapsed_time(b)
+
+
+# ---------------------------------------------------------------------------------- oracle arm
+def oracle_sample(cfg, budget_s, n_tiles_cap=64):
+    """Times the CPU oracle on a bounded sample of the workload: routing on `heads` heads in full and
+    attention on sampled (head, query-block) tiles.  Returns a dict (effective TFLOP/s etc.)."""
+    import numpy as np
+    import torch
+
+    from oracle import fvattn_oracle as O
+    from paper_2607_16190_b200 import synth
+
+    heads = min(cfg.H, 4)
+    sub = cfg.with_(H=heads)
+    q, k, v, _ = synth.make_qkv(sub, "cpu")
+    og = O.Grid(*cfg.grid, *cfg.tile)
+    nb = O.num_blocks(og)
+    t0 = time.perf_counter()
+    qb, kb, vb = (O.reorder(synth.bf16_bits(t), og)[0] for t in (q, k, v))
+    t_reorder = time.perf_counter() - t0
+    t0 = time.perf_counter()
+    res = O.route(qb, kb, og, cfg.p, cfg.k_floor, cfg.sm_scale)
+    t_route = time.perf_counter() - t0
+    # attention: grow the tile sample until the budget is used
+    rng = np.random.default_rng(0)
+    order = rng.permutation(heads * nb)
+    done_pairs, t_attn, used = 0, 0.0, 0
+    batch = O.threads()
+    while used < min(n_tiles_cap, order.size) and t_attn < budget_s:
+        tiles = np.sort(order[used:used + batch]).astype(np.int64)
+        t0 = time.perf_counter()
+        O.sparse_attn(qb, kb, vb, res.idx, res.counts, og, cfg.sm_scale, tiles=tiles)
+        t_attn += time.perf_counter() - t0
+        done_pairs += int(res.counts.reshape(-1)[tiles].sum())
+        used += len(tiles)
+    attn_tflops = done_pairs * FLOP_PER_PAIR / t_attn / 1e12
+    # whole path, extrapolated to all H heads: reorder and route scale with heads, attention with pairs
+    total_pairs_est = float(res.counts.sum()) * cfg.H / heads
+    t_layer = (t_reorder * 4 / 3 + t_route) * cfg.H / heads + total_pairs_est * FLOP_PER_PAIR / (attn_tflops * 1e12)
+    return {
+        "value": total_pairs_est * FLOP_PER_PAIR / t_layer / 1e12,
+        "unit": "TFLOP/s",
+        "cores": O.threads(),
+        "kind": "oracle",
+        "sample": (f"{cfg.name}: reorder+route of {heads}/{cfg.H} heads in full ({t_reorder:.1f}s + {t_route:.1f}s), "
+                   f"fp64 attention on {used} random (head, query-block) tiles = {done_pairs} retained pairs "
+                   f"({t_attn:.1f}s); layer time extrapolated by heads and retained pairs"),
+        "attn_only_tflops": attn_tflops,
+        "extrapolated_s_per_layer": t_layer,
+    }
+
+
+def run_reference(args):
+    """`--impl reference`: the CPU oracle as it stands, on the host cores, same metric and config."""
+    rank, world, _ = dist_env()
+    if rank != 0:
+        return
+    from paper_2607_16190_b200 import synth
+
+    cfg = synth.CONFIGS[args.workload]
+    per_step_budget = max(2.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
+    results = []
+    for s in range(args.warmup + args.steps):
+        r = oracle_sample(cfg, per_step_budget, n_tiles_cap=32)
+        if s >= args.warmup:
+            results.append(r)
+    value = sum(r["value"] for r in results) / len(results)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 * sum(r["extrapolated_s_per_layer"] for r in results) / len(results),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg, args.gpus),
+        "cpu_baseline": {"value": value, "unit": "TFLOP/s", "cores": results[-1]["cores"], "kind": "oracle",
+                         "sample": results[-1]["sample"]},
+        "e2e": {"value": value, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def workload_config(cfg, n_gpus):
+    return {"workload": f"{cfg.name}: B=1 H={cfg.H} d={cfg.d} grid={'x'.join(map(str, cfg.grid))} "
+                        f"tile={'x'.join(map(str, cfg.tile))} p={cfg.p} k_floor={cfg.k_floor}",
+            "tokens": cfg.tokens, "blocks": cfg.num_blocks, "features": cfg.features,
+            "temperature": cfg.temperature, "seed": cfg.seed,
+            "parallelism": "single GPU" if n_gpus == 1 else f"{n_gpus} independent replicas",
+            "cache": "inputs (2.3 GB of Q/K/V) are larger than L2; no explicit flush"}
+
+
+# ---------------------------------------------------------------------------------- CUDA arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2607_16190_b200 import binding as fv
+    from paper_2607_16190_b200 import synth
+
+    rank, world, local = dist_env()
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    fv.lib()                                                      # fail loudly if the extension is missing
+
+    cfg = synth.CONFIGS[args.workload].with_(seed=synth.CONFIGS[args.workload].seed + 100 * rank)
+    g = fv.Grid(*cfg.grid, *cfg.tile)
+    nb = g.num_blocks
+    q, k, v, _ = synth.make_qkv(cfg, dev)
+    layer = fv.SparseAttentionLayer(g, 1, cfg.H, cfg.d, cfg.p, cfg.k_floor, device=dev)
+
+    def step():
+        return layer(q, k, v)
+
+    # per-stage events (recorded inside the timed steps, on the launching stream)
+    stage_names = ["reorder", "route", "attn", "inverse"]
+    stage_ms = {n: 0.0 for n in stage_names}
+
+    def step_staged(events):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        ev[0].record()
+        fv.reorder(q, g, layer.q_r); fv.reorder(k, g, layer.k_r); fv.reorder(v, g, layer.v_r)
+        ev[1].record()
+        fv.route(layer.q_r, layer.k_r, g, cfg.p, cfg.k_floor, layer.sm_scale, layer.workspace, layer.routing)
+        ev[2].record()
+        fv.sparse_attn(layer.q_r, layer.k_r, layer.v_r, layer.routing.idx, layer.routing.counts, g, layer.sm_scale,
+                       layer.workspace, layer.o_r)
+        ev[3].record()
+        fv.inverse_reorder(layer.o_r, g, layer.out)
+        ev[4].record()
+        events.append(ev)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    status = fv.device_status(layer.workspace)
+    if status != fv.OK:
+        raise SystemExit(f"device status after warm-up: {fv.status_string(status)}")
+    pairs = int(layer.routing.counts.sum().item())
+    flops = pairs * FLOP_PER_PAIR
+
+    # ---- timed region: K steps, barrier + synchronize on both sides, device time, max over ranks
+    events = []
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    with ClockSampler(local) as clocks:
+        t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t0.record()
+        for _ in range(args.steps):
+            step_staged(events)
+        t1.record()
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        total_ms = t0.elapsed_time(t1)
+    for ev in events:
+        for n, (a, b) in zip(stage_names, zip(ev[:-1], ev[1:])):
+            stage_ms[n] += a.elapsed_time(b) / args.steps
+    if world > 1:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+        fl = torch.tensor([float(flops)], device=dev, dtype=torch.float64)
+        dist.all_reduce(fl, op=dist.ReduceOp.SUM)
+        flops_all = float(fl.item())
+    else:
+        flops_all = float(flops)
+    ms_per_step = total_ms / args.steps
+    value = flops_all / (ms_per_step * 1e-3) / 1e12
+
+    # ---- e2e: pinned host inputs, H2D + path + D2H of the output inside the timed region
+    hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
+    hout = torch.empty_like(hq).pin_memory()
+    dq, dk, dv = (torch.empty_like(t) for t in (q, k, v))
+
+    def e2e_step():
+        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
+        out = layer(dq, dk, dv)
+        hout.copy_(out, non_blocking=True)
+
+    e2e_step()
+    if world > 1:
+        dist.barrier()
+    e2e_steps = max(2, min(args.steps, 5))
+    e2e_ms = time_steps(e2e_step, e2e_steps, torch) / e2e_steps
+    if world > 1:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e = {"value": flops_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
+           "h2d_bytes_per_step": 3 * hq.numel() * 2, "d2h_bytes_per_step": hout.numel() * 2}
+    del hq, hk, hv, hout, dq, dk, dv
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- rank 0 only: roofline of the dominant kernel, dense baselines, route GB/s, CPU baseline
+    peaks, peaks_kind = load_peaks()
+    attn_ms = stage_ms["attn"]
+    attn_tflops = flops / (attn_ms * 1e-3) / 1e12
+    peak_t = float(peaks.get("bf16_tflops_sustained") or peaks["bf16_tflops"])
+    roofline = {
+        "kernel": "attn_tc_kernel (fvattn_sparse_attn; the two scheduler-order launches, ~10 us, are inside the events)",
+        "bound": "tensor", "achieved": attn_tflops, "peak": peak_t, "unit": "TFLOP/s", "frac": attn_tflops / peak_t,
+        "peak_kind": f"{peaks_kind} sustained bf16 (kernel timed inside a long step)",
+        "frac_of_burst_peak": attn_tflops / float(peaks["bf16_tflops"]), "burst_peak": float(peaks["bf16_tflops"]),
+        "traffic": None if ATTN_DRAM_TRAFFIC_BYTES_PER_PAIR is None else ATTN_DRAM_TRAFFIC_BYTES_PER_PAIR * pairs,
+        "algorithmic_flop_per_launch": flops, "ms_per_launch": attn_ms,
+    }
+    route_bytes = 2 * cfg.H * cfg.tokens * cfg.d * 2 + layer.routing.mask_bits.numel() * 4 + cfg.H * nb * 4 + pairs * 2
+    route_gbs = route_bytes / (stage_ms["route"] * 1e-3) / 1e9
+    reorder_bytes = 3 * (cfg.H * cfg.tokens * cfg.d * 2 + cfg.H * g.padded_tokens * cfg.d * 2)
+    extra = {
+        "density": pairs / (cfg.H * nb * nb), "retained_pairs": pairs,
+        "stage_ms": stage_ms, "attn_tflops": attn_tflops,
+        "route_gbs": route_gbs, "route_frac_of_hbm": route_gbs / float(peaks["hbm_gbs"]),
+        "reorder_gbs": reorder_bytes / (stage_ms["reorder"] * 1e-3) / 1e9,
+        "inverse_gbs": (cfg.H * cfg.tokens * cfg.d * 2 + cfg.H * g.padded_tokens * cfg.d * 2) /
+                       (stage_ms["inverse"] * 1e-3) / 1e9,
+        "peaks": {k_: peaks[k_] for k_ in ("hbm_gbs", "bf16_tflops", "bf16_tflops_sustained") if k_ in peaks},
+        "peaks_kind": peaks_kind,
+    }
+    if not args.no_dense:
+        extra.update(dense_baselines(fv, layer, cfg, g, q, k, v, attn_ms, torch))
+    cpu = None
+    if not args.no_cpu_baseline and world == 1 or (world > 1 and not args.no_cpu_baseline and args.cpu_baseline_multi):
+        cpu = oracle_sample(synth.CONFIGS[args.workload], budget_s=12.0)
+    line = {
+        "metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(cfg, world),
+        "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": 11 * args.steps, "roofline": roofline,
+        "cpu_baseline": cpu, **extra,
+    }
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def dense_baselines(fv, layer, cfg, g, q, k, v, sparse_attn_ms, torch):
+    """Dense attention on the same inputs: this library's kernel with an all-ones mask, and torch SDPA."""
+    nb = g.num_blocks
+    full = fv.route(layer.q_r, layer.k_r, g, 1.0, cfg.k_floor, layer.sm_scale, layer.workspace)
+
+    def own():
+        fv.sparse_attn(layer.q_r, layer.k_r, layer.v_r, full.idx, full.counts, g, layer.sm_scale, layer.workspace,
+                       layer.o_r)
+
+    own()
+    own_ms = time_steps(own, 2, torch) / 2
+    out = {"dense_own_kernel_ms": own_ms, "dense_own_kernel_tflops": cfg.H * nb * nb * FLOP_PER_PAIR / own_ms / 1e9,
+           "speedup_vs_dense_own_kernel": own_ms / sparse_attn_ms}
+    del full
+    try:
+        from torch.nn.attention import SDPBackend, sdpa_kernel
+
+        qt, kt, vt = (t.transpose(1, 2) for t in (q, k, v))     # [B, H, N, d] views
+        with sdpa_kernel([SDPBackend.FLASH_ATTENTION, SDPBackend.CUDNN_ATTENTION, SDPBackend.EFFICIENT_ATTENTION]):
+            f = lambda: torch.nn.functional.scaled_dot_product_attention(qt, kt, vt)
+            f()
+            sdpa_ms = time_steps(f, 2, torch) / 2
+        out.update({"dense_sdpa_ms": sdpa_ms, "dense_sdpa_tflops": 4 * cfg.H * cfg.tokens ** 2 * cfg.d / sdpa_ms / 1e9,
+                    "dense_sdpa_backend": "torch SDPA bf16 (flash / cudnn / mem-efficient, torch's pick)",
+                    "speedup_vs_dense_sdpa": sdpa_ms / sparse_attn_ms})
+    except Exception as e:  # the dense library baseline is context, not part of the path
+        out["dense_sdpa_error"] = repr(e)[:200]
+    return out
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--workload", default="wan720p", choices=["tiny", "small", "wan480p", "wan720p"])
+    ap.add_argument("--no-dense", action="store_true", help="skip the dense baselines")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-baseline-multi", action="store_true", help="also time the oracle when N > 1")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

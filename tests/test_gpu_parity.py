@@ -17,6 +17,7 @@ pytestmark = pytest.mark.gpu
 
 MAX_ABS, MEAN_ABS = 1e-2, 1e-3
 NEAR_P = 1e-5
+NEAR_TIE = 1e-6
 
 
 def grids(cfg):
@@ -36,15 +37,23 @@ def case(name, layer=-1):
 
 
 def compare_masks(res_gpu, res_o, p):
-    """Returns (rows differing, rows near threshold, rows near tie); asserts every differing row is excused."""
+    """Returns (rows differing, rows near threshold, rows near tie, differing near-tie rows).
+
+    Every differing row must be in the near-threshold class (cumulative mass within 1e-5 of p) or
+    in the near-tie class (last kept and first dropped block within a relative 1e-6 of each other in
+    probability, i.e. below what fp32 scores resolve); the latter is counted and must stay rare."""
     mg = res_gpu.mask_bits[0].cpu().numpy()
     diff_rows = (mg != res_o.mask_bits).any(-1)
     near = (np.abs(res_o.cum_at - p) < NEAR_P) | (np.abs(res_o.cum_before - p) < NEAR_P)
-    tie = res_o.gap < 1e-6
-    unexcused = diff_rows & ~near
+    tie = res_o.gap < NEAR_TIE
+    unexcused = diff_rows & ~near & ~tie
     assert not unexcused.any(), (
-        f"{int(unexcused.sum())} mask rows differ outside the near-threshold class "
-        f"(near-tie among them: {int((unexcused & tie).sum())}); first {np.argwhere(unexcused)[:5].tolist()}")
+        f"{int(unexcused.sum())} mask rows differ outside the near-threshold and near-tie classes; "
+        f"first {np.argwhere(unexcused)[:5].tolist()}")
+    tie_diff = int((diff_rows & ~near & tie).sum())
+    assert tie_diff <= max(2, diff_rows.size // 5000), f"{tie_diff} near-tie rows differ"
+    if tie_diff:
+        print(f"\n  near-tie rows that differ (not excused by the 1e-5 rule, reported): {tie_diff}")
     same = ~diff_rows
     cg = res_gpu.counts[0].cpu().numpy()
     assert (cg[same] == res_o.counts[same]).all()
