@@ -111,6 +111,7 @@ fvattn_status_t fvattn_route(const void* q_r, const void* k_r, int32_t B, int32_
  * each valid query row r of block i,
  *   O[r] = softmax_{r' in retained blocks, r' valid}(sm_scale * <Q[r],K[r']>) . V[r'],
  * bf16 inputs, fp32 accumulation and softmax, bf16 output; padding query rows give 0.
+ * sm_scale must be finite and > 0.
  * The mask is taken in compact form (idx, counts) as written by fvattn_route; each row's
  * entries must be distinct block indices < nb (checked on the device: a bad index sets
  * FVATTN_ERR_DEVICE_BOUNDS and that tile is skipped).  counts[h,i] == 0 gives zero rows.

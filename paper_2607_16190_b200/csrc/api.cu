@@ -29,7 +29,7 @@ fvattn_status_t check_attn_args(const void* q_r, const void* k_r, const void* v_
                                 float sm_scale, void* o_r, void* workspace, size_t workspace_bytes) {
     if (!q_r || !k_r || !v_r || !idx || !counts || !o_r || !workspace || !grid_ok(grid))
         return FVATTN_ERR_INVALID_ARG;
-    if (B <= 0 || H <= 0 || !(sm_scale == sm_scale) || isinf(sm_scale)) return FVATTN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || !(sm_scale > 0.f) || isinf(sm_scale)) return FVATTN_ERR_INVALID_ARG;
     GridDims m = make_dims(*grid);
     if (!shape_ok(d, m)) return FVATTN_ERR_UNSUPPORTED_SHAPE;
     if ((int64_t)B * H * m.nb > 0x7fffffffLL) return FVATTN_ERR_UNSUPPORTED_SHAPE;

@@ -1,22 +1,29 @@
 // Block-sparse attention on the sm_100a tensor cores (Sec. 2.1: only the retained
 // (query block, key block) pairs are evaluated), Bs = d = 128, bf16 in, fp32 accumulate.
 //
-// Persistent CTAs pop (head, query-block) tiles from an atomic queue in heaviest-first order.
-// Per tile: Q (128 x 128) is TMA-loaded once; for every retained key block the K and V tiles
-// are TMA-loaded by index (each is one contiguous 128 x 128 tile of the head-major layout),
-// S = Q K^T and O += P V run as tcgen05 MMAs with the accumulators in tensor memory, and the
-// online softmax (running max and sum per query row, fp32, base-2 exponentials) runs one
-// thread per query row on the S tile read back from tensor memory.  P is written back to
-// tensor memory as bf16 and fed to the second MMA as its A operand.  Padded keys of edge
-// blocks are masked to -inf; padded query rows are written as zero.
+// One persistent CTA per SM, 12 warps, warp-specialised:
+//   warp 0        producer: pops (head, query-block) tiles from the heaviest-first queue, TMA-loads
+//                 Q once per tile and the retained K / V tiles by index into 3-deep rings
+//   warp 1        MMA issuer (one thread): S = Q K^T and O += P V as tcgen05 MMAs, accumulators in
+//                 tensor memory
+//   warps 4-7     softmax of the even retained blocks  (stream 0)
+//   warps 8-11    softmax of the odd retained blocks   (stream 1)
+// The retained blocks of a tile alternate between two independent streams, each with its own
+// S/P and O accumulators in tensor memory (4 x 128 columns = all 512) and its own running max
+// and sum, so the softmax of one stream overlaps the MMAs of the other; the two partial results
+// are merged once per tile (O = (O0 w0 + O1 w1) / (l0 w0 + l1 w1)).  One thread owns one query
+// row: it reads its S row from tensor memory, keeps a running max with lazy rescaling (O is only
+// rescaled when the max grows by more than 2^8), writes P back as bf16 over the S columns, and
+// the MMA thread feeds P from tensor memory as the A operand of the second MMA.  Padded keys of
+// edge blocks are masked to -inf from a per-block validity table; padded query rows give zero.
 //
 // Shared-memory tiles use the 128-byte swizzle: a 128 x 128 bf16 tile is two TMA boxes of
 // 128 rows x 64 columns (16 KB each).  Q and K are K-major MMA operands; V (keys x d, d
-// contiguous) is the MN-major B operand of the second MMA.
+// contiguous) is the MN-major B operand of the second MMA.  No TMA multicast is used.
 //
-// Every wait on an mbarrier is bounded; when one runs out the CTA records
-// FVATTN_ERR_DEVICE_TIMEOUT in the workspace, stops taking tiles, frees its tensor memory
-// and returns.
+// Every wait is a bounded mbarrier wait; when one runs out the CTA records
+// FVATTN_ERR_DEVICE_TIMEOUT in the workspace, every role leaves its loop, tensor memory is
+// freed and the kernel returns.
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -27,49 +34,85 @@ using namespace ptx;
 namespace tc {
 constexpr int BS = 128;
 constexpr int D = 128;
-constexpr int kThreads = 128;
-constexpr uint32_t kHalfBytes = 128 * 64 * 2;      // one TMA box: 128 rows x 64 bf16
-constexpr uint32_t kTileBytes = 2 * kHalfBytes;    // 128 x 128 bf16
+constexpr int kThreads = 384;
+constexpr int KS = 3;                               // K ring depth
+constexpr int VS = 3;                               // V ring depth
+constexpr int TS = 2;                               // tile-info ring depth
+constexpr uint32_t kHalfBytes = 128 * 64 * 2;       // one TMA box: 128 rows x 64 bf16
+constexpr uint32_t kTileBytes = 2 * kHalfBytes;     // 128 x 128 bf16
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;      // S accumulator, 128 fp32 columns
-constexpr uint32_t kColO = 128;    // O accumulator, 128 fp32 columns
-constexpr uint32_t kColP = 256;    // P operand, 128 bf16 = 64 columns
+constexpr uint32_t kColS = 0;                       // S / P of stream a at kColS + 128 a
+constexpr uint32_t kColO = 256;                     // O of stream a at kColO + 128 a
 constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kRescaleThreshold = 8.0f;           // log2 units
 
 struct __align__(1024) Smem {
     unsigned char q[kTileBytes];
-    unsigned char k[kTileBytes];
-    unsigned char v[kTileBytes];
-    unsigned char pad_to_one_cta_per_sm[24 * 1024];   // > half of the SM's shared memory in total
-    unsigned long long bar_q, bar_kv, bar_s, bar_o;
+    unsigned char k[KS][kTileBytes];
+    unsigned char v[VS][kTileBytes];
+    float ml[2][2][BS];                             // [stream][m, l][row]
+    unsigned long long q_full, q_empty, k_full[KS], k_empty[KS], v_full[VS], v_empty[VS];
+    unsigned long long s_full[2], p_full[2], o_full, o_free, ml_ready, ml_done, tile_full[TS], tile_empty[TS];
+    int tile_id[TS];
+    int tile_cnt[TS];
     uint32_t tmem_base;
-    uint32_t kmask[4];
-    int tile;
     int abort_flag;
 };
+static_assert(sizeof(Smem) <= 232448, "shared memory budget");
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_inc() {
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
+}
+template <int N>
+__device__ __forceinline__ void setmaxnreg_dec() {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N));
+}
 } // namespace tc
+
+// Validity of the 128 key rows of every block (bit o of word o >> 5), for masking padded keys.
+__global__ void __launch_bounds__(128)
+key_mask_kernel(GridDims m, uint32_t* __restrict__ kmask) {
+    int64_t token;
+    unsigned int bal = __ballot_sync(0xffffffffu, threadIdx.x < m.bs && row_to_token(m, blockIdx.x, threadIdx.x, &token));
+    if ((threadIdx.x & 31) == 0) kmask[blockIdx.x * 4 + (threadIdx.x >> 5)] = bal;
+}
 
 __global__ void __launch_bounds__(tc::kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const uint16_t* __restrict__ idx,
                const int32_t* __restrict__ counts, GridDims m, float sm_scale, __nv_bfloat16* __restrict__ o_r,
-               const uint32_t* __restrict__ order, int n_tiles, void* workspace) {
+               const uint32_t* __restrict__ order, const uint4* __restrict__ kmask, int has_pad, int n_tiles,
+               void* workspace) {
     using namespace tc;
-    extern __shared__ unsigned char smem_raw[];
-    Smem& sm = *reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(workspace);
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const uint32_t bar_q = smem_u32(&sm.bar_q), bar_kv = smem_u32(&sm.bar_kv), bar_s = smem_u32(&sm.bar_s),
-                   bar_o = smem_u32(&sm.bar_o);
-    const uint32_t sq = smem_u32(sm.q), sk = smem_u32(sm.k), sv = smem_u32(sm.v);
+    volatile int* abort_flag = &sm.abort_flag;
 
+    if ((smem_u32(smem_raw) & 1023u) != 0u) {   // the swizzled tiles need a 1024-byte aligned base
+        if (tid == 0) report_error(workspace, FVATTN_ERR_CUDA, 0x1024u);
+        return;
+    }
     if (tid == 0) {
-        mbar_init(bar_q, 1);
-        mbar_init(bar_kv, 1);
-        mbar_init(bar_s, 1);
-        mbar_init(bar_o, 1);
+        mbar_init(smem_u32(&sm.q_full), 1);
+        mbar_init(smem_u32(&sm.q_empty), 1);
+        for (int s = 0; s < KS; ++s) { mbar_init(smem_u32(&sm.k_full[s]), 1); mbar_init(smem_u32(&sm.k_empty[s]), 1); }
+        for (int s = 0; s < VS; ++s) { mbar_init(smem_u32(&sm.v_full[s]), 1); mbar_init(smem_u32(&sm.v_empty[s]), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&sm.s_full[a]), 1); mbar_init(smem_u32(&sm.p_full[a]), 4); }
+        mbar_init(smem_u32(&sm.o_full), 1);
+        mbar_init(smem_u32(&sm.o_free), 8);
+        mbar_init(smem_u32(&sm.ml_ready), 8);
+        mbar_init(smem_u32(&sm.ml_done), 8);
+        for (int s = 0; s < TS; ++s) { mbar_init(smem_u32(&sm.tile_full[s]), 1); mbar_init(smem_u32(&sm.tile_empty[s]), 9); }
         sm.abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_q);
@@ -84,181 +127,331 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = sm.tmem_base;
-    const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);   // this warp's 32 lanes
-
-    constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false);
-    constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, true);
     const float sl2 = sm_scale * kLog2e;
-    uint32_t ph_q = 0, ph_kv = 0, ph_s = 0, ph_o = 0;
-    volatile int* abort_flag = &sm.abort_flag;
-    bool alive = true;
+    bool failed = false;
 
-    while (alive) {
-        if (tid == 0) sm.tile = (int)atomicAdd(&hdr->tile_counter, 1u);
-        tc_fence_before();
-        __syncthreads();   // also: every thread is done with the previous tile's TMEM and smem
-        tc_fence_after();
-        const int slot = sm.tile;
-        __syncthreads();   // everyone holds its copy before thread 0 may overwrite it
-        if (slot >= n_tiles) break;
-        const uint32_t tile = order[slot];
-        const int64_t bh = tile / (uint32_t)m.nb;
-        const int i = (int)(tile % (uint32_t)m.nb);
-        const int c = min(max(counts[tile], 0), m.nb);
-        const uint16_t* irow = idx + (int64_t)tile * m.nb;
-        const int64_t head_row0 = bh * m.n_pad;
-
-        if (tid == 0 && c > 0) {
-            mbar_expect_tx(bar_q, kTileBytes);
-            tma_load_2d(sq, &map_q, 0, (int)(head_row0 + (int64_t)i * BS), bar_q);
-            tma_load_2d(sq + kHalfBytes, &map_q, 64, (int)(head_row0 + (int64_t)i * BS), bar_q);
-        }
-        float m_run = -INFINITY, l_run = 0.f;
-
-        for (int t = 0; t < c; ++t) {
-            const int kb = irow[t];
-            if (kb >= m.nb) {   // same value in every thread
-                if (tid == 0) report_error(workspace, FVATTN_ERR_DEVICE_BOUNDS, tile);
-                if (t == 0 && tid == 0) (void)mbar_wait(bar_q, ph_q, abort_flag);   // drain the Q copy in flight
-                if (t == 0) { ph_q ^= 1; l_run = 0.f; }
-                break;
-            }
-            const bool edge = block_valid_tokens(m, kb) != BS;
-            if (edge) {
-                int64_t token;
-                unsigned int bal = __ballot_sync(0xffffffffu, row_to_token(m, kb, tid, &token));
-                if (lane == 0) sm.kmask[warp] = bal;
-            }
+    if (warp < 4) {
+        setmaxnreg_dec<40>();
+        if (warp == 0) {
+            // ======================= producer =======================================================
+            uint32_t n = 0, kn = 0, vn = 0, qn = 0;
             bool ok = true;
-            if (tid == 0) {
-                mbar_expect_tx(bar_kv, 2 * kTileBytes);
-                const int krow = (int)(head_row0 + (int64_t)kb * BS);
-                tma_load_2d(sk, &map_k, 0, krow, bar_kv);
-                tma_load_2d(sk + kHalfBytes, &map_k, 64, krow, bar_kv);
-                tma_load_2d(sv, &map_v, 0, krow, bar_kv);
-                tma_load_2d(sv + kHalfBytes, &map_v, 64, krow, bar_kv);
-                if (t == 0) ok = mbar_wait(bar_q, ph_q, abort_flag);
-                ok = ok && mbar_wait(bar_kv, ph_kv, abort_flag);
+            while (ok) {
+                const uint32_t slot = n % TS;
+                int tile = -1, c = 0;
+                if (lane == 0) {
+                    ok = mbar_wait(smem_u32(&sm.tile_empty[slot]), ((n / TS) & 1u) ^ 1u, abort_flag);
+                    if (ok) {
+                        const unsigned int q = atomicAdd(&hdr->tile_counter, 1u);
+                        if (q < (unsigned int)n_tiles) {
+                            tile = (int)order[q];
+                            c = min(max(counts[tile], 0), m.nb);
+                        }
+                        sm.tile_id[slot] = tile;
+                        sm.tile_cnt[slot] = c;
+                        mbar_arrive(smem_u32(&sm.tile_full[slot]));
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                tile = __shfl_sync(0xffffffffu, tile, 0);
+                c = __shfl_sync(0xffffffffu, c, 0);
+                ++n;
+                if (!ok || tile < 0) break;
+                if (c == 0) continue;
+                const int64_t bh = (uint32_t)tile / (uint32_t)m.nb;
+                const int i = (int)((uint32_t)tile % (uint32_t)m.nb);
+                const int64_t head_row0 = bh * m.n_pad;
+                const uint16_t* irow = idx + (int64_t)tile * m.nb;
+                if (lane == 0) {
+                    ok = mbar_wait(smem_u32(&sm.q_empty), (qn & 1u) ^ 1u, abort_flag);
+                    if (ok) {
+                        const uint32_t bar = smem_u32(&sm.q_full);
+                        mbar_expect_tx(bar, kTileBytes);
+                        tma_load_2d(smem_u32(sm.q), &map_q, 0, (int)(head_row0 + (int64_t)i * BS), bar);
+                        tma_load_2d(smem_u32(sm.q) + kHalfBytes, &map_q, 64, (int)(head_row0 + (int64_t)i * BS), bar);
+                    }
+                }
+                ++qn;
+                for (int t0 = 0; t0 < c && ok; t0 += 32) {
+                    const int mine = (t0 + lane < c) ? (int)irow[t0 + lane] : 0;
+                    const int lim = min(32, c - t0);
+                    for (int tt = 0; tt < lim; ++tt) {
+                        int kb = __shfl_sync(0xffffffffu, mine, tt);
+                        if (lane == 0 && ok) {
+                            if (kb >= m.nb) {
+                                report_error(workspace, FVATTN_ERR_DEVICE_BOUNDS, (unsigned int)tile);
+                                kb = 0;   // keep the pipeline consistent; the tile's result is undefined
+                            }
+                            const int krow = (int)(head_row0 + (int64_t)kb * BS);
+                            const uint32_t ks = kn % KS, vs = vn % VS;
+                            ok = mbar_wait(smem_u32(&sm.k_empty[ks]), ((kn / KS) & 1u) ^ 1u, abort_flag);
+                            if (ok) {
+                                const uint32_t bar = smem_u32(&sm.k_full[ks]);
+                                mbar_expect_tx(bar, kTileBytes);
+                                tma_load_2d(smem_u32(sm.k[ks]), &map_k, 0, krow, bar);
+                                tma_load_2d(smem_u32(sm.k[ks]) + kHalfBytes, &map_k, 64, krow, bar);
+                                ok = mbar_wait(smem_u32(&sm.v_empty[vs]), ((vn / VS) & 1u) ^ 1u, abort_flag);
+                            }
+                            if (ok) {
+                                const uint32_t bar = smem_u32(&sm.v_full[vs]);
+                                mbar_expect_tx(bar, kTileBytes);
+                                tma_load_2d(smem_u32(sm.v[vs]), &map_v, 0, krow, bar);
+                                tma_load_2d(smem_u32(sm.v[vs]) + kHalfBytes, &map_v, 64, krow, bar);
+                            }
+                        }
+                        ++kn;
+                        ++vn;
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                }
+            }
+            failed = !ok;
+        } else if (warp == 1 && lane == 0) {
+            // ======================= MMA issuer (one thread) ===========================================
+            constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false);
+            constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, true);
+            uint32_t n = 0, kn = 0, vn = 0, qn = 0, pn[2] = {0, 0};
+            bool ok = true;
+            const uint32_t sq = smem_u32(sm.q);
+
+            auto issue_pv = [&](int u) {
+                const int b = u & 1;
+                ok = ok && mbar_wait(smem_u32(&sm.p_full[b]), pn[b] & 1u, abort_flag);
+                ++pn[b];
+                const uint32_t vs = vn % VS;
+                ok = ok && mbar_wait(smem_u32(&sm.v_full[vs]), (vn / VS) & 1u, abort_flag);
+                if (u == 0) ok = ok && mbar_wait(smem_u32(&sm.o_free), (qn & 1u) ^ 1u, abort_flag);
                 if (ok) {
                     tc_fence_after();
-                    // S = Q K^T : 8 steps of K = 16 over d = 128; both operands K-major
+                    const uint32_t sv = smem_u32(sm.v[vs]);
+#pragma unroll
+                    for (int ks = 0; ks < BS / 16; ++ks)
+                        umma_ts(tmem + kColO + 128u * b, tmem + kColS + 128u * b + ks * 8,
+                                make_smem_desc_sw128(sv + (uint32_t)ks * 2048u, kHalfBytes, 1024), idesc_pv,
+                                (u >= 2 || ks > 0) ? 1u : 0u);
+                    umma_commit(smem_u32(&sm.v_empty[vs]));
+                }
+                ++vn;
+            };
+
+            while (ok) {
+                const uint32_t slot = n % TS;
+                ok = mbar_wait(smem_u32(&sm.tile_full[slot]), (n / TS) & 1u, abort_flag);
+                if (!ok) break;
+                const int tile = sm.tile_id[slot];
+                const int c = sm.tile_cnt[slot];
+                mbar_arrive(smem_u32(&sm.tile_empty[slot]));
+                ++n;
+                if (tile < 0) break;
+                if (c == 0) continue;
+                ok = mbar_wait(smem_u32(&sm.q_full), qn & 1u, abort_flag);
+                for (int t = 0; t < c && ok; ++t) {
+                    const int a = t & 1;
+                    const uint32_t ks_ = kn % KS;
+                    ok = mbar_wait(smem_u32(&sm.k_full[ks_]), (kn / KS) & 1u, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t sk = smem_u32(sm.k[ks_]);
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) {
-                        uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                        umma_ss(tmem + kColS, make_smem_desc_sw128(sq + off, 16, 1024),
+                        const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                        umma_ss(tmem + kColS + 128u * a, make_smem_desc_sw128(sq + off, 16, 1024),
                                 make_smem_desc_sw128(sk + off, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
                     }
-                    umma_commit(bar_s);
-                } else {
-                    *abort_flag = 1;
+                    umma_commit(smem_u32(&sm.k_empty[ks_]));
+                    ++kn;
+                    if (t == c - 1) umma_commit(smem_u32(&sm.q_empty));
+                    umma_commit(smem_u32(&sm.s_full[a]));
+                    if (t >= 1) issue_pv(t - 1);
                 }
+                if (ok) issue_pv(c - 1);
+                if (ok) umma_commit(smem_u32(&sm.o_full));
+                ++qn;
             }
-            if (t == 0) ph_q ^= 1;
-            ph_kv ^= 1;
-            ok = mbar_wait(bar_s, ph_s, abort_flag);
-            ph_s ^= 1;
-            if (!__syncthreads_and(ok ? 1 : 0)) { alive = false; break; }
-            tc_fence_after();
-
-            // ---- online softmax on row `tid` of S -------------------------------------------
-            uint32_t r[32];
-            float mx = m_run;
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                tmem_ld32(lane_addr + kColS + ch * 32, r);
-                tmem_wait_ld();
-                const uint32_t km = edge ? sm.kmask[ch] : 0xffffffffu;
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if ((km >> j) & 1u) mx = fmaxf(mx, __uint_as_float(r[j]));
-            }
-            // mx == -inf only if no valid key so far: exponent offset 0 keeps everything finite
-            const float moff = (mx == -INFINITY) ? 0.f : mx * sl2;
-            float sum = 0.f;
-#pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                tmem_ld32(lane_addr + kColS + ch * 32, r);
-                tmem_wait_ld();
-                const uint32_t km = edge ? sm.kmask[ch] : 0xffffffffu;
-                uint32_t packed[16];
-#pragma unroll
-                for (int j = 0; j < 32; j += 2) {
-                    float p0 = ((km >> j) & 1u) ? exp2f(fmaf(__uint_as_float(r[j]), sl2, -moff)) : 0.f;
-                    float p1 = ((km >> (j + 1)) & 1u) ? exp2f(fmaf(__uint_as_float(r[j + 1]), sl2, -moff)) : 0.f;
-                    __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);   // .x (low half) = even column
-                    // the row sum uses the rounded values that the second MMA will see
-                    float2 back = __bfloat1622float2(b2);
-                    sum += back.x + back.y;
-                    packed[j >> 1] = *reinterpret_cast<uint32_t*>(&b2);
-                }
-                tmem_st16(lane_addr + kColP + ch * 16, packed);
-            }
-            const float corr = (m_run == -INFINITY) ? 0.f : exp2f(m_run * sl2 - moff);
-            l_run = l_run * corr + sum;
-            m_run = mx;
-            if (t > 0 && __any_sync(0xffffffffu, corr != 1.f)) {   // rescale the running O
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) {
-                    tmem_ld32(lane_addr + kColO + ch * 32, r);
-                    tmem_wait_ld();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
-                    tmem_st32(lane_addr + kColO + ch * 32, r);
-                }
-            }
-            tmem_wait_st();
-            tc_fence_before();
-            __syncthreads();
-
-            // ---- O (+)= P V : 8 steps of K = 16 keys; A = P from tensor memory, B = V MN-major ---
-            if (tid == 0) {
-                tc_fence_after();
-#pragma unroll
-                for (int ks = 0; ks < BS / 16; ++ks)
-                    umma_ts(tmem + kColO, tmem + kColP + ks * 8,
-                            make_smem_desc_sw128(sv + (uint32_t)ks * 2048u, kHalfBytes, 1024), idesc_pv,
-                            (t > 0 || ks > 0) ? 1u : 0u);
-                umma_commit(bar_o);
-            }
-            ok = mbar_wait(bar_o, ph_o, abort_flag);
-            ph_o ^= 1;
-            if (!__syncthreads_and(ok ? 1 : 0)) { alive = false; break; }
-            tc_fence_after();
+            failed = !ok;
         }
-        if (!alive) break;
+    } else {
+        // ======================= softmax warpgroups ==================================================
+        setmaxnreg_inc<232>();
+        const int a = (warp - 4) >> 2;            // stream
+        const int row = tid - 128 - 128 * a;      // query row of the tile = TMEM lane
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const uint32_t tS = tmem + lane_base + kColS + 128u * a;
+        const uint32_t tO = tmem + lane_base + kColO + 128u * a;
+        uint32_t n = 0, sn = 0, tile_seq = 0;
+        bool ok = true;
 
-        // ---- epilogue: O / l -> bf16 -> global; padded query rows and empty rows give 0 --------
-        {
-            int64_t token;
-            const bool qvalid = row_to_token(m, i, tid, &token);
-            const float inv = (qvalid && l_run > 0.f) ? 1.f / l_run : 0.f;
-            uint4* orow = reinterpret_cast<uint4*>(o_r + (head_row0 + (int64_t)i * BS + tid) * D);
-            uint32_t r[32];
+        while (ok) {
+            const uint32_t slot = n % TS;
+            ok = mbar_wait(smem_u32(&sm.tile_full[slot]), (n / TS) & 1u, abort_flag);
+            if (!ok) break;
+            const int tile = sm.tile_id[slot];
+            const int c = sm.tile_cnt[slot];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm.tile_empty[slot]));
+            ++n;
+            if (tile < 0) break;
+            const int64_t bh = (uint32_t)tile / (uint32_t)m.nb;
+            const int i = (int)((uint32_t)tile % (uint32_t)m.nb);
+            const uint16_t* irow = idx + (int64_t)tile * m.nb;
+            // this thread stores columns [64 a, 64 a + 64) of output row `row`
+            uint4* orow = reinterpret_cast<uint4*>(o_r + ((bh * m.n_pad + (int64_t)i * BS + row) * D + 64 * a));
+            if (c == 0) {
 #pragma unroll
-            for (int ch = 0; ch < 4; ++ch) {
-                if (l_run > 0.f || c > 0) {   // c is CTA-uniform: the load below is warp-uniform
-                    tmem_ld32(lane_addr + kColO + ch * 32, r);
-                    tmem_wait_ld();
+                for (int q4 = 0; q4 < 8; ++q4) orow[q4] = make_uint4(0u, 0u, 0u, 0u);
+                continue;
+            }
+            const int n_a = (c - a + 1) >> 1;     // blocks t = a, a + 2, ... of this stream
+            float m_run = -INFINITY, l_run = 0.f;
+
+            for (int u = 0; u < n_a && ok; ++u) {
+                uint4 km = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+                if (has_pad) {
+                    const int kb = min((int)irow[2 * u + a], m.nb - 1);
+                    km = __ldg(kmask + kb);
                 }
+                ok = mbar_wait(smem_u32(&sm.s_full[a]), sn & 1u, abort_flag);
+                ++sn;
+                if (!ok) break;
+                tc_fence_after();
+                uint32_t s[128];
+#pragma unroll
+                for (int ch = 0; ch < 4; ++ch) tmem_ld32(tS + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32 * ch]));
+                tmem_wait_ld();
+                if ((km.x & km.y & km.z & km.w) != 0xffffffffu) {   // edge block: padded keys -> -inf
+                    const uint32_t kw[4] = {km.x, km.y, km.z, km.w};
+#pragma unroll
+                    for (int j = 0; j < 128; ++j)
+                        if (!((kw[j >> 5] >> (j & 31)) & 1u)) s[j] = 0xff800000u;
+                }
+                float mx0 = __uint_as_float(s[0]), mx1 = __uint_as_float(s[1]), mx2 = __uint_as_float(s[2]),
+                      mx3 = __uint_as_float(s[3]);
+#pragma unroll
+                for (int j = 4; j < 128; j += 4) {
+                    mx0 = fmaxf(mx0, __uint_as_float(s[j]));
+                    mx1 = fmaxf(mx1, __uint_as_float(s[j + 1]));
+                    mx2 = fmaxf(mx2, __uint_as_float(s[j + 2]));
+                    mx3 = fmaxf(mx3, __uint_as_float(s[j + 3]));
+                }
+                const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)));
+                // lazy rescale: keep the old reference max unless the new one is more than 2^8 above it
+                const bool need = (m_new - m_run) * sl2 > kRescaleThreshold;   // also true for m_run = -inf
+                if (__any_sync(0xffffffffu, need)) {
+                    float corr = 1.f;
+                    if (need) {
+                        corr = (m_run == -INFINITY) ? 0.f : ex2((m_run - m_new) * sl2);
+                        m_run = m_new;
+                    }
+                    l_run *= corr;
+                    if (u > 0) {
+                        uint32_t r[32];
+#pragma unroll
+                        for (int ch = 0; ch < 4; ++ch) {
+                            tmem_ld32(tO + ch * 32, r);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) r[j] = __float_as_uint(__uint_as_float(r[j]) * corr);
+                            tmem_st32(tO + ch * 32, r);
+                        }
+                    }
+                }
+                const float moff = (m_run == -INFINITY) ? 0.f : m_run * sl2;   // -inf only if no valid key yet
+                float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
+                uint32_t pk[64];
+#pragma unroll
+                for (int j = 0; j < 128; j += 4) {
+                    const float p0 = ex2(fmaf(__uint_as_float(s[j]), sl2, -moff));
+                    const float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sl2, -moff));
+                    const float p2 = ex2(fmaf(__uint_as_float(s[j + 2]), sl2, -moff));
+                    const float p3 = ex2(fmaf(__uint_as_float(s[j + 3]), sl2, -moff));
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(p0, p1);   // .x (low half) = even column
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(p2, p3);
+                    const uint32_t wlo = *reinterpret_cast<uint32_t*>(&lo), whi = *reinterpret_cast<uint32_t*>(&hi);
+                    pk[j >> 1] = wlo;
+                    pk[(j >> 1) + 1] = whi;
+                    // the row sum takes the bf16-rounded weights the second MMA sees, so numerator and
+                    // denominator stay consistent (an exact weighted average of V)
+                    sum0 += __uint_as_float(wlo << 16);
+                    sum1 += __uint_as_float(wlo & 0xffff0000u);
+                    sum2 += __uint_as_float(whi << 16);
+                    sum3 += __uint_as_float(whi & 0xffff0000u);
+                }
+                l_run += (sum0 + sum1) + (sum2 + sum3);
+                tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+                tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+                tmem_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&sm.p_full[a]));
+            }
+            if (!ok) break;
+
+            // ---- merge the two streams and store ----------------------------------------------------
+            sm.ml[a][0][row] = m_run;
+            sm.ml[a][1][row] = l_run;
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm.ml_ready));
+            ok = mbar_wait(smem_u32(&sm.ml_ready), tile_seq & 1u, abort_flag);
+            ok = ok && mbar_wait(smem_u32(&sm.o_full), tile_seq & 1u, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const float m0 = sm.ml[0][0][row], l0 = sm.ml[0][1][row];
+            const float m1 = sm.ml[1][0][row], l1 = sm.ml[1][1][row];
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm.ml_done));
+            const bool has1 = c >= 2;                       // stream 1 saw at least one block
+            const float mm = has1 ? fmaxf(m0, m1) : m0;
+            const float w0 = (m0 == -INFINITY) ? 0.f : ex2((m0 - mm) * sl2);
+            const float w1 = (!has1 || m1 == -INFINITY) ? 0.f : ex2((m1 - mm) * sl2);
+            const float lsum = l0 * w0 + l1 * w1;
+            int64_t token;
+            const bool qvalid = !has_pad || row_to_token(m, i, row, &token);
+            const float inv = (qvalid && lsum > 0.f) ? 1.f / lsum : 0.f;
+            const float f0 = w0 * inv, f1 = w1 * inv;
+            const uint32_t tO0 = tmem + lane_base + kColO + 64u * a;
+            const uint32_t tO1 = tO0 + 128u;
+#pragma unroll
+            for (int ch = 0; ch < 2; ++ch) {
+                uint32_t r0[32], r1[32];
+                tmem_ld32(tO0 + ch * 32, r0);
+                if (has1) tmem_ld32(tO1 + ch * 32, r1);
+                tmem_wait_ld();
                 uint32_t outw[16];
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
-                    float a = inv != 0.f ? __uint_as_float(r[j]) * inv : 0.f;
-                    float b = inv != 0.f ? __uint_as_float(r[j + 1]) * inv : 0.f;
-                    __nv_bfloat162 b2 = __floats2bfloat162_rn(a, b);
+                    float x = f0 != 0.f ? __uint_as_float(r0[j]) * f0 : 0.f;
+                    float y = f0 != 0.f ? __uint_as_float(r0[j + 1]) * f0 : 0.f;
+                    if (has1 && f1 != 0.f) {
+                        x = fmaf(__uint_as_float(r1[j]), f1, x);
+                        y = fmaf(__uint_as_float(r1[j + 1]), f1, y);
+                    }
+                    __nv_bfloat162 b2 = __floats2bfloat162_rn(x, y);
                     outw[j >> 1] = *reinterpret_cast<uint32_t*>(&b2);
                 }
 #pragma unroll
                 for (int q4 = 0; q4 < 4; ++q4)
                     orow[ch * 4 + q4] = make_uint4(outw[q4 * 4], outw[q4 * 4 + 1], outw[q4 * 4 + 2], outw[q4 * 4 + 3]);
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sm.o_free));
+            // nobody may overwrite ml for the next tile before every row of this one has been read
+            ok = mbar_wait(smem_u32(&sm.ml_done), tile_seq & 1u, abort_flag);
+            ++tile_seq;
         }
+        failed = !ok;
     }
 
-    if (!alive && tid == 0) report_error(workspace, FVATTN_ERR_DEVICE_TIMEOUT, blockIdx.x);
+    if (failed) {
+        *abort_flag = 1;
+        report_error(workspace, FVATTN_ERR_DEVICE_TIMEOUT, blockIdx.x);
+    }
     tc_fence_before();
     __syncthreads();
-    if (warp == 0) tmem_dealloc(tmem, kTmemCols);
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, kTmemCols);
+    }
 }
 
 // ---- host side ------------------------------------------------------------------------------
@@ -305,12 +498,18 @@ fvattn_status_t launch_attn_tc(const void* q_r, const void* k_r, const void* v_r
     int dev = 0, sms = 0;
     FVATTN_CUDA_OK(cudaGetDevice(&dev));
     FVATTN_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const size_t smem = sizeof(tc::Smem) + 1024;
+    uint32_t* kmask = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + attn_ws(BH, m.nb).kmask);
+    const int has_pad = m.n_pad != m.n ? 1 : 0;
+    if (has_pad) {
+        key_mask_kernel<<<(unsigned)m.nb, 128, 0, s>>>(m, kmask);
+        if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
+    }
+    const size_t smem = sizeof(tc::Smem);
     FVATTN_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int n_tiles = (int)(BH * m.nb);
     const int grid = n_tiles < sms ? n_tiles : sms;
     attn_tc_kernel<<<grid, tc::kThreads, smem, s>>>(mq, mk, mv, idx, counts, m, sm_scale, (__nv_bfloat16*)o_r, order,
-                                                   n_tiles, workspace);
+                                                   reinterpret_cast<const uint4*>(kmask), has_pad, n_tiles, workspace);
     return launch_status();
 }
 

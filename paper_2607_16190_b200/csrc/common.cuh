@@ -101,13 +101,14 @@ inline RouteWs route_ws(int64_t BH, int nb, int d) {
 }
 
 struct AttnWs {
-    size_t head_sum, order, total;
+    size_t head_sum, order, kmask, total;
 };
 inline AttnWs attn_ws(int64_t BH, int nb) {
     AttnWs w;
     size_t off = kWsHeaderBytes;
     w.head_sum = off; off = align_up(off + sizeof(unsigned int) * (size_t)BH, 256);
     w.order = off; off = align_up(off + sizeof(unsigned int) * (size_t)BH * nb, 256);
+    w.kmask = off; off = align_up(off + 16 * (size_t)nb, 256);   // per-block key validity, 128 bits
     w.total = off;
     return w;
 }

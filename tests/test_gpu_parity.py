@@ -250,7 +250,9 @@ def test_tensor_core_kernel_agrees_with_cuda_core_kernel():
     res = fv.route(c["q_r"], c["k_r"], g, 0.7, 1, cfg.sm_scale, ws)
     a = fv.sparse_attn(c["q_r"], c["k_r"], c["v_r"], res.idx, res.counts, g, cfg.sm_scale, ws)
     b = fv.sparse_attn_simt(c["q_r"], c["k_r"], c["v_r"], res.idx, res.counts, g, cfg.sm_scale, ws)
-    assert (a.float() - b.float()).abs().max().item() <= 1e-2
+    # both kernels round their fp32 result to bf16: they may land one bf16 ulp (2^-7 relative) apart
+    diff = (a.float() - b.float()).abs()
+    assert (diff <= 5e-3 + a.float().abs() * 2.0 ** -7).all(), diff.max().item()
 
 
 def test_attention_edge_cases():
