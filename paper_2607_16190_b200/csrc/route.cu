@@ -31,16 +31,23 @@ pool_kernel(const uint4* __restrict__ q_r, const uint4* __restrict__ k_r, float*
 
     const int v = threadIdx.x % VPR;
     const int rg = threadIdx.x / VPR;
+    const bool full = block_valid_tokens(m, blk) == m.bs;   // no padding rows in this block
+    // issue every load of this thread before the first add: 8 x 16 B in flight per thread
+    constexpr int kPasses = 8;
+    uint4 raw[kPasses];
+#pragma unroll
+    for (int it = 0; it < kPasses; ++it) {
+        const int o = rg + it * RG;
+        int64_t token;
+        const bool take = o < m.bs && (full || row_to_token(m, blk, o, &token));   // padding rows take no part
+        raw[it] = take ? __ldg(x + (int64_t)o * VPR + v) : make_uint4(0u, 0u, 0u, 0u);
+    }
     float acc[8];
 #pragma unroll
     for (int e = 0; e < 8; ++e) acc[e] = 0.f;
-
-#pragma unroll 4
-    for (int o = rg; o < m.bs; o += RG) {
-        int64_t token;
-        if (!row_to_token(m, blk, o, &token)) continue;   // padding rows take no part in the mean
-        uint4 raw = __ldg(x + (int64_t)o * VPR + v);
-        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
+#pragma unroll
+    for (int it = 0; it < kPasses; ++it) {
+        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw[it]);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             float2 f = __bfloat1622float2(h2[e]);
@@ -276,6 +283,144 @@ select_kernel(const float* __restrict__ scores, int nb, int n2, int score_stride
     if (tid == 0) counts[row] = c;
 }
 
+// One warp per (head, query block) row, nb <= 1024: the row lives in registers (E = ceil(nb/32)
+// entries per lane, block j = lane + 32 e).  Instead of sorting, the warp bisects on the 32-bit
+// order-preserving image of the score: the smallest threshold t such that the blocks with
+// key <= t hold mass >= p and number at least max(1, min(k_floor, nb)) is the key of the last
+// kept block, so {key <= t} is exactly the prefix the descending sort would have kept.  Blocks
+// whose score equals the threshold's are admitted in index order one at a time (the tie rule).
+// The ballot of the keep flags over entry e is the mask word for blocks 32e..32e+31, and its
+// prefix pop-counts give the ascending compact index list.
+constexpr int kSelWarpsPerCta = 8;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+template <int E>
+__global__ void __launch_bounds__(kSelWarpsPerCta * 32)
+select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int score_stride, float p, int k_floor,
+                   uint32_t* __restrict__ mask_bits, int32_t* __restrict__ counts, uint16_t* __restrict__ idx) {
+    const int lane = threadIdx.x & 31;
+    const int64_t row = (int64_t)blockIdx.x * kSelWarpsPerCta + (threadIdx.x >> 5);
+    if (row >= n_rows) return;
+    const float* srow = scores + row * score_stride;
+
+    float prob[E];
+    uint32_t key[E];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const int j = lane + 32 * e;
+        const float sc = (j < nb) ? srow[j] + 0.0f : -INFINITY;   // -0 -> +0: equal scores, equal keys
+        prob[e] = sc;
+        mx = fmaxf(mx, sc);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float z = 0.f;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const int j = lane + 32 * e;
+        uint32_t u = __float_as_uint(prob[e]);
+        u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+        key[e] = (j < nb) ? ~u : 0xffffffffu;                   // ascending key = descending score
+        const float ex = (j < nb) ? expf(prob[e] - mx) : 0.f;
+        prob[e] = ex;
+        z += ex;
+    }
+    z = warp_sum(z);
+#pragma unroll
+    for (int e = 0; e < E; ++e) prob[e] = prob[e] / z;
+
+    const int need_cnt = max(1, min(k_floor, nb));
+    uint32_t thr = 0xffffffffu;          // p >= 1 keeps everything
+    int r_ties = 1 << 30;                // how many blocks with key == thr are kept (index order)
+    if (p < 1.0f) {
+        uint32_t lo = 0u, hi = 0xffffffffu;
+#pragma unroll 1
+        while (lo < hi) {
+            const uint32_t mid = lo + ((hi - lo) >> 1);
+            float mass = 0.f;
+            int cnt = 0;
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const bool in = key[e] <= mid;
+                mass += in ? prob[e] : 0.f;
+                cnt += in ? 1 : 0;
+            }
+            mass = warp_sum(mass);
+            cnt = warp_sum(cnt);
+            if (mass >= p && cnt >= need_cnt) hi = mid; else lo = mid + 1;
+        }
+        thr = hi;
+        // blocks tied with the threshold score: admit them one by one, lowest index first
+        float mass_lt = 0.f, p_tie = 0.f;
+        int cnt_lt = 0, n_tie = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const bool lt = key[e] < thr, eq = key[e] == thr && (lane + 32 * e) < nb;
+            mass_lt += lt ? prob[e] : 0.f;
+            cnt_lt += lt ? 1 : 0;
+            n_tie += eq ? 1 : 0;
+            p_tie = eq ? prob[e] : p_tie;
+        }
+        mass_lt = warp_sum(mass_lt);
+        cnt_lt = warp_sum(cnt_lt);
+        n_tie = warp_sum(n_tie);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) p_tie = fmaxf(p_tie, __shfl_xor_sync(0xffffffffu, p_tie, o));
+        if (n_tie > 1) {
+            float cum = mass_lt;
+            int r = 0;
+            while (r < n_tie) {
+                cum += p_tie;
+                ++r;
+                if (cum >= p && cnt_lt + r >= need_cnt) break;
+            }
+            r_ties = r;
+        }
+    }
+
+    // materialise
+    uint32_t* mrow = mask_bits + row * ((nb + 31) / 32);
+    uint16_t* irow = idx + row * nb;
+    int base = 0, ties_seen = 0;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const int j = lane + 32 * e;
+        const bool eq = key[e] == thr && j < nb;
+        const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
+        const int tie_rank = ties_seen + __popc(eq_ballot & ((1u << lane) - 1u));
+        ties_seen += __popc(eq_ballot);
+        const bool keep = j < nb && (key[e] < thr || (eq && tie_rank < r_ties));
+        const uint32_t word = __ballot_sync(0xffffffffu, keep);
+        if (32 * e < nb) {
+            if (lane == 0) mrow[e] = word;
+            if (keep) irow[base + __popc(word & ((1u << lane) - 1u))] = (uint16_t)j;
+        }
+        base += __popc(word);
+    }
+    if (lane == 0) counts[row] = base;
+}
+
+template <int E>
+static fvattn_status_t launch_select_warp(const float* scores, int nb, int64_t n_rows, int score_stride, float p,
+                                          int k_floor, uint32_t* mask_bits, int32_t* counts, uint16_t* idx,
+                                          cudaStream_t s) {
+    const unsigned ctas = (unsigned)((n_rows + kSelWarpsPerCta - 1) / kSelWarpsPerCta);
+    select_warp_kernel<E><<<ctas, kSelWarpsPerCta * 32, 0, s>>>(scores, nb, n_rows, score_stride, p, k_floor,
+                                                                  mask_bits, counts, idx);
+    return launch_status();
+}
+
 __global__ void __launch_bounds__(256)
 head_load_kernel(const int32_t* __restrict__ counts, int nb, float* __restrict__ head_load) {
     __shared__ unsigned int red[8];
@@ -315,14 +460,26 @@ fvattn_status_t launch_route(const void* q_r, const void* k_r, int64_t BH, int d
                                                                    sm_scale);
     if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
 
-    int n2 = 32;
-    while (n2 < m.nb) n2 <<= 1;
-    size_t smem = (size_t)n2 * (8 + 4 + 4) + 2 * sizeof(uint32_t) * (size_t)(n2 / 32);
-    if (smem > 48 * 1024)
+    if (m.nb <= 1024) {
+        const int e = (m.nb + 31) / 32;
+        const int64_t n_rows = BH * m.nb;
+        fvattn_status_t st;
+#define FVATTN_SEL_CASE(E_) \
+    if (e <= E_) st = launch_select_warp<E_>(scores, m.nb, n_rows, w.score_stride, p, k_floor, mask_bits, counts, idx, s); else
+        FVATTN_SEL_CASE(1) FVATTN_SEL_CASE(4) FVATTN_SEL_CASE(8) FVATTN_SEL_CASE(12) FVATTN_SEL_CASE(16)
+        FVATTN_SEL_CASE(20) FVATTN_SEL_CASE(24) FVATTN_SEL_CASE(28)
+        st = launch_select_warp<32>(scores, m.nb, n_rows, w.score_stride, p, k_floor, mask_bits, counts, idx, s);
+#undef FVATTN_SEL_CASE
+        if (st != FVATTN_OK) return st;
+    } else {
+        int n2 = 2048;
+        while (n2 < m.nb) n2 <<= 1;
+        size_t smem = (size_t)n2 * (8 + 4 + 4) + 2 * sizeof(uint32_t) * (size_t)(n2 / 32);
         FVATTN_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    select_kernel<<<(unsigned)(BH * m.nb), kSelThreads, smem, s>>>(scores, m.nb, n2, w.score_stride, p, k_floor,
-                                                                  mask_bits, counts, idx);
-    if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
+        select_kernel<<<(unsigned)(BH * m.nb), kSelThreads, smem, s>>>(scores, m.nb, n2, w.score_stride, p, k_floor,
+                                                                      mask_bits, counts, idx);
+        if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
+    }
 
     if (head_load) {
         head_load_kernel<<<(unsigned)BH, 256, 0, s>>>(counts, m.nb, head_load);
