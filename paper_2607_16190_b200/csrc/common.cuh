@@ -86,15 +86,16 @@ __device__ __forceinline__ void report_error(void* workspace, unsigned int statu
 inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
 struct RouteWs {
-    size_t qbar, kbar, scores, total;
+    size_t qsplit, ksplit, scores, total;
     int score_stride; // floats per score row
 };
+// qsplit / ksplit: the pooled means as three bf16 parts (hi, mid, lo), [3][BH][nb][d] each.
 inline RouteWs route_ws(int64_t BH, int nb, int d) {
     RouteWs w;
     w.score_stride = (nb + 3) / 4 * 4;
     size_t off = kWsHeaderBytes;
-    w.qbar = off; off = align_up(off + sizeof(float) * (size_t)BH * nb * d, 256);
-    w.kbar = off; off = align_up(off + sizeof(float) * (size_t)BH * nb * d, 256);
+    w.qsplit = off; off = align_up(off + 3 * sizeof(__nv_bfloat16) * (size_t)BH * nb * d, 256);
+    w.ksplit = off; off = align_up(off + 3 * sizeof(__nv_bfloat16) * (size_t)BH * nb * d, 256);
     w.scores = off; off = align_up(off + sizeof(float) * (size_t)BH * nb * w.score_stride, 256);
     w.total = off;
     return w;

@@ -1,127 +1,259 @@
 // Top-p block routing with a Top-k floor (Sec. 2.1, Sec. 3.1, Eq. 1).
 //
-//   pool_kernel    block means of Q and K over valid rows            HBM-bound: reads Q, K once
-//   score_kernel   s = sm_scale * qbar kbar^T per head, fp32 FFMA    small fp32 GEMM, L2-resident
-//   select_kernel  per (head, query block): softmax, sort by (score desc, index asc),
-//                  prefix-sum mass cut at p, floor, bit mask + counts + compact index list
-//   head_load_kernel  L_h = mean_i counts (Eq. 1)
+//   pool_kernel        block means of Q and K over valid rows: persistent CTAs stream the blocks
+//                      through shared memory with bulk async copies (HBM-bound, reads Q and K once)
+//                      and write every mean as three bf16 parts (hi + mid + lo = the fp32 mean)
+//   score_tc_kernel    s = sm_scale * qbar kbar^T per head on the tensor cores: the six leading
+//                      part products (hi hi, hi mid, mid hi, hi lo, mid mid, lo hi) accumulate in
+//                      fp32 in tensor memory, which reproduces the fp32 product to its last bits
+//   select_warp_kernel per (head, query block): softmax, threshold search on the ordered score
+//                      keys, mass cut at p, floor, ties by index -> bit mask, counts, index list
+//   head_load_kernel   L_h = mean_i counts (Eq. 1)
 //
-// All arithmetic that decides the mask is fp32 with fp32 accumulation in a fixed order
-// (no tensor cores, no fast-math), so the mask is reproducible run to run and differs from
-// an fp64 evaluation only on rows whose cumulative mass sits within rounding of p.
+// The mask decision is deterministic run to run: pooled sums, exponentials and the fixed-point
+// masses are computed in a fixed order, and differs from an fp64 evaluation only on rows whose
+// cumulative mass sits within rounding of p or whose boundary scores tie to fp32 precision.
 #include "common.cuh"
+#include "sm100_ptx.cuh"
 
 namespace fvattn {
 
+using namespace ptx;
+
 // ------------------------------------------------------------------------------------ pool
 constexpr int kPoolThreads = 256;
+constexpr int kPoolStages = 4;
+
+// x = hi + mid + lo exactly (3 x 8 significant bits), each part a bf16.
+__device__ __forceinline__ void split3(float x, __nv_bfloat16& hi, __nv_bfloat16& mid, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(x);
+    const float r1 = x - __bfloat162float(hi);
+    mid = __float2bfloat16_rn(r1);
+    lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+}
 
 template <int D>
 __global__ void __launch_bounds__(kPoolThreads)
-pool_kernel(const uint4* __restrict__ q_r, const uint4* __restrict__ k_r, float* __restrict__ qbar,
-            float* __restrict__ kbar, GridDims m) {
+pool_kernel(const uint4* __restrict__ q_r, const uint4* __restrict__ k_r, __nv_bfloat16* __restrict__ qsplit,
+            __nv_bfloat16* __restrict__ ksplit, GridDims m, int64_t BH, void* workspace) {
     constexpr int VPR = D / 8;                // 16-byte vectors per row
-    constexpr int RG = kPoolThreads / VPR;    // rows in flight per pass
-    __shared__ float partial[RG][D];
+    constexpr int RG = kPoolThreads / VPR;    // rows added per pass
+    constexpr int kPasses = 8;                // covers Bs <= 8 * RG
+    extern __shared__ __align__(128) unsigned char pool_smem[];
+    const uint32_t block_bytes = (uint32_t)m.bs * D * 2;
+    float* partial = reinterpret_cast<float*>(pool_smem + (size_t)kPoolStages * block_bytes);   // [2][RG][D]
+    unsigned short* vcount = reinterpret_cast<unsigned short*>(partial + 2 * RG * D);           // [nb] valid rows
+    __shared__ unsigned long long full[kPoolStages];
+    __shared__ int abort_flag;
 
-    const int blk = blockIdx.x;
-    const int64_t bh = blockIdx.y;
-    const uint4* x = (blockIdx.z == 0 ? q_r : k_r) + (bh * m.n_pad + (int64_t)blk * m.bs) * VPR;
-    float* out = (blockIdx.z == 0 ? qbar : kbar) + (bh * m.nb + blk) * D;
+    const int tid = threadIdx.x;
+    const int64_t per_tensor = BH * m.nb;
+    const int64_t n_items = 2 * per_tensor;                         // item = (tensor, head, block), memory order
+    const int64_t first = blockIdx.x, stride = gridDim.x;
+    const int64_t my_items = first < n_items ? (n_items - first + stride - 1) / stride : 0;
+    const int64_t part_stride = per_tensor * D;                     // elements between the hi / mid / lo planes
 
-    const int v = threadIdx.x % VPR;
-    const int rg = threadIdx.x / VPR;
-    const bool full = block_valid_tokens(m, blk) == m.bs;   // no padding rows in this block
-    // issue every load of this thread before the first add: 8 x 16 B in flight per thread
-    constexpr int kPasses = 8;
-    uint4 raw[kPasses];
+    for (int b = tid; b < m.nb; b += kPoolThreads) vcount[b] = (unsigned short)block_valid_tokens(m, b);
+    if (tid == 0) {
+        for (int s = 0; s < kPoolStages; ++s) mbar_init(smem_u32(&full[s]), 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    auto issue = [&](int64_t k) {                                   // thread 0 only
+        const int64_t item = first + k * stride;
+        const int64_t rest = item >= per_tensor ? item - per_tensor : item;
+        const uint4* src = (item >= per_tensor ? k_r : q_r) + rest * (int64_t)m.bs * VPR;
+        const int s = (int)(k % kPoolStages);
+        const uint32_t bar = smem_u32(&full[s]);
+        mbar_expect_tx(bar, block_bytes);
+        bulk_load_1d(smem_u32(pool_smem + (size_t)s * block_bytes), src, block_bytes, bar);
+    };
+    if (tid == 0)
+        for (int64_t k = 0; k < kPoolStages - 1 && k < my_items; ++k) issue(k);
+
+    const int v = tid % VPR, rg = tid / VPR;
+    // offsets of this thread's rows inside a tile, packed (t, y, x): they do not depend on the block
+    uint32_t row_off[kPasses];
 #pragma unroll
     for (int it = 0; it < kPasses; ++it) {
         const int o = rg + it * RG;
-        int64_t token;
-        const bool take = o < m.bs && (full || row_to_token(m, blk, o, &token));   // padding rows take no part
-        raw[it] = take ? __ldg(x + (int64_t)o * VPR + v) : make_uint4(0u, 0u, 0u, 0u);
+        row_off[it] = (uint32_t)(o / (m.tX * m.tY)) | ((uint32_t)((o / m.tX) % m.tY) << 10) | ((uint32_t)(o % m.tX) << 20);
     }
-    float acc[8];
+    int blk = (int)(first % m.nb);
+    const int blk_step = (int)(stride % m.nb);
+    int stage = 0;
+    uint32_t phase = 0;
+    for (int64_t k = 0; k < my_items; ++k) {
+        // the stage refilled here was read during iteration k - 1, which every thread has left
+        if (tid == 0 && k + kPoolStages - 1 < my_items) issue(k + kPoolStages - 1);
+        const int64_t item = first + k * stride;
+        const int64_t rest = item >= per_tensor ? item - per_tensor : item;
+        const int nvalid = vcount[blk];
+        bool ok = mbar_wait(smem_u32(&full[stage]), phase, &abort_flag);
+        const uint4* tile = reinterpret_cast<const uint4*>(pool_smem + (size_t)stage * block_bytes);
+        float acc[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+        for (int e = 0; e < 8; ++e) acc[e] = 0.f;
+        if (ok) {
+            // valid extents of an edge block; a whole block takes every row
+            uint32_t vt = 1024, vy = 1024, vx = 1024;
+            if (nvalid != m.bs) {
+                const int bx = blk % m.nX, by = (blk / m.nX) % m.nY, bt = blk / (m.nX * m.nY);
+                vt = min(m.tT, m.T - bt * m.tT); vy = min(m.tY, m.Y - by * m.tY); vx = min(m.tX, m.X - bx * m.tX);
+            }
 #pragma unroll
-    for (int it = 0; it < kPasses; ++it) {
-        const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw[it]);
+            for (int it = 0; it < kPasses; ++it) {
+                const int o = rg + it * RG;
+                const uint32_t ro = row_off[it];
+                const bool take = o < m.bs && (ro & 1023u) < vt && ((ro >> 10) & 1023u) < vy && (ro >> 20) < vx;
+                if (take) {                                          // padding rows take no part in the mean
+                    const uint4 raw = tile[o * VPR + v];
+                    const __nv_bfloat162* h2 = reinterpret_cast<const __nv_bfloat162*>(&raw);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-            float2 f = __bfloat1622float2(h2[e]);
-            acc[2 * e] += f.x;
-            acc[2 * e + 1] += f.y;
+                    for (int e = 0; e < 4; ++e) {
+                        float2 f = __bfloat1622float2(h2[e]);
+                        acc[2 * e] += f.x;
+                        acc[2 * e + 1] += f.y;
+                    }
+                }
+            }
+        } else {
+            abort_flag = 1;
         }
-    }
+        float* part = partial + (size_t)(k & 1) * RG * D;
 #pragma unroll
-    for (int e = 0; e < 8; ++e) partial[rg][v * 8 + e] = acc[e];
-    __syncthreads();
-    if (threadIdx.x < D) {
-        float s = 0.f;
+        for (int e = 0; e < 8; ++e) part[rg * D + v * 8 + e] = acc[e];
+        if (!__syncthreads_and(ok ? 1 : 0)) {
+            if (tid == 0) report_error(workspace, FVATTN_ERR_DEVICE_TIMEOUT, 0x9001u);
+            break;
+        }
+        if (tid < D) {
+            float sum = 0.f;
 #pragma unroll
-        for (int g = 0; g < RG; ++g) s += partial[g][threadIdx.x];
-        out[threadIdx.x] = s / (float)block_valid_tokens(m, blk);
+            for (int g = 0; g < RG; ++g) sum += part[g * D + tid];
+            __nv_bfloat16 hi, mid, lo;
+            split3(sum / (float)nvalid, hi, mid, lo);
+            __nv_bfloat16* out = (item >= per_tensor ? ksplit : qsplit) + rest * D + tid;
+            out[0] = hi;
+            out[part_stride] = mid;
+            out[2 * part_stride] = lo;
+        }
+        blk += blk_step;
+        if (blk >= m.nb) blk -= m.nb;
+        if (++stage == kPoolStages) { stage = 0; phase ^= 1u; }
     }
 }
 
 // ----------------------------------------------------------------------------------- scores
-constexpr int kScoreTile = 64;
-constexpr int kScoreK = 32;
+// One CTA per 128 x 128 tile of one head's score matrix.  The six operand tiles (three parts of
+// the 128 query-block means, three of the 128 key-block means) are TMA-loaded with the 128-byte
+// swizzle (rows past nb are zero-filled by the copy engine), one thread issues the 6 x d/16
+// tcgen05 MMAs, and the four warps read the fp32 accumulator from tensor memory, scale it and
+// store their rows.  Small products are accumulated first.
+namespace sc {
+constexpr int kThreads = 128;
+constexpr uint32_t kHalfBytes = 128 * 64 * 2;
+}
 
-__global__ void __launch_bounds__(256)
-score_kernel(const float* __restrict__ qbar, const float* __restrict__ kbar, float* __restrict__ scores, int nb,
-             int d, int score_stride, float sm_scale) {
-    __shared__ __align__(16) float As[kScoreK][kScoreTile + 4];
-    __shared__ __align__(16) float Bs[kScoreK][kScoreTile + 4];
-    const int64_t bh = blockIdx.z;
-    const int i0 = blockIdx.y * kScoreTile, j0 = blockIdx.x * kScoreTile;
-    const float* A = qbar + bh * (int64_t)nb * d;
-    const float* Bm = kbar + bh * (int64_t)nb * d;
-    const int tx = threadIdx.x % 16, ty = threadIdx.x / 16;
-    float acc[4][4];
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-        for (int b = 0; b < 4; ++b) acc[a][b] = 0.f;
+template <int D>
+__global__ void __launch_bounds__(sc::kThreads, 1)
+score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                float* __restrict__ scores, int nb, int BH, int score_stride, float sm_scale, void* workspace) {
+    using namespace sc;
+    constexpr uint32_t kPartBytes = 128 * D * 2;                  // one 128 x d operand tile
+    constexpr int kHalves = D / 64;
+    extern __shared__ __align__(1024) unsigned char sc_smem[];
+    unsigned char* a_parts = sc_smem;                              // [3][kPartBytes]
+    unsigned char* b_parts = sc_smem + 3 * kPartBytes;             // [3][kPartBytes]
+    __shared__ unsigned long long bar_full, bar_done;
+    __shared__ uint32_t tmem_slot;
+    __shared__ int abort_flag;
 
-    for (int k0 = 0; k0 < d; k0 += kScoreK) {
-        // 64 rows x 32 k per operand; thread -> (row = t / 8 + 32 * r, 4 consecutive k)
-#pragma unroll
-        for (int r = 0; r < 2; ++r) {
-            int row = threadIdx.x / 8 + 32 * r;
-            int kk = (threadIdx.x % 8) * 4;
-            float4 va = make_float4(0.f, 0.f, 0.f, 0.f), vb = va;
-            if (i0 + row < nb) va = *reinterpret_cast<const float4*>(A + (int64_t)(i0 + row) * d + k0 + kk);
-            if (j0 + row < nb) vb = *reinterpret_cast<const float4*>(Bm + (int64_t)(j0 + row) * d + k0 + kk);
-            As[kk + 0][row] = va.x; As[kk + 1][row] = va.y; As[kk + 2][row] = va.z; As[kk + 3][row] = va.w;
-            Bs[kk + 0][row] = vb.x; Bs[kk + 1][row] = vb.y; Bs[kk + 2][row] = vb.z; Bs[kk + 3][row] = vb.w;
-        }
-        __syncthreads();
-#pragma unroll
-        for (int kk = 0; kk < kScoreK; ++kk) {
-            float4 a4 = *reinterpret_cast<const float4*>(&As[kk][ty * 4]);
-            float4 b4 = *reinterpret_cast<const float4*>(&Bs[kk][tx * 4]);
-            float av[4] = {a4.x, a4.y, a4.z, a4.w};
-            float bv[4] = {b4.x, b4.y, b4.z, b4.w};
-#pragma unroll
-            for (int a = 0; a < 4; ++a)
-#pragma unroll
-                for (int b = 0; b < 4; ++b) acc[a][b] = fmaf(av[a], bv[b], acc[a][b]);
-        }
-        __syncthreads();
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int j0 = blockIdx.x * 128, i0 = blockIdx.y * 128, bh = blockIdx.z;
+    if ((smem_u32(sc_smem) & 1023u) != 0u) {
+        if (tid == 0) report_error(workspace, FVATTN_ERR_CUDA, 0x1025u);
+        return;
     }
+    if (tid == 0) {
+        mbar_init(smem_u32(&bar_full), 1);
+        mbar_init(smem_u32(&bar_done), 1);
+        abort_flag = 0;
+        fence_barrier_init();
+    }
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&tmem_slot), 128);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_slot;
+
+    bool ok = true;
+    if (tid == 0) {
+        const uint32_t bar = smem_u32(&bar_full);
+        mbar_expect_tx(bar, 6 * kPartBytes);
+        for (int part = 0; part < 3; ++part)
+            for (int h = 0; h < kHalves; ++h) {
+                tma_load_3d(smem_u32(a_parts) + part * kPartBytes + h * kHalfBytes, &map_q, 64 * h, i0, part * BH + bh, bar);
+                tma_load_3d(smem_u32(b_parts) + part * kPartBytes + h * kHalfBytes, &map_k, 64 * h, j0, part * BH + bh, bar);
+            }
+        ok = mbar_wait(bar, 0, &abort_flag);
+        if (ok) {
+            tc_fence_after();
+            constexpr uint32_t idesc = make_idesc_bf16(128, 128, false);
+            // (query part, key part), smallest products first
+            const int combo[6][2] = {{0, 2}, {1, 1}, {2, 0}, {0, 1}, {1, 0}, {0, 0}};
+            bool first = true;
 #pragma unroll
-    for (int a = 0; a < 4; ++a) {
-        int i = i0 + ty * 4 + a;
-        if (i >= nb) continue;
-        float* out = scores + (bh * nb + i) * (int64_t)score_stride;
+            for (int cidx = 0; cidx < 6; ++cidx) {
+                const uint32_t sa = smem_u32(a_parts) + combo[cidx][0] * kPartBytes;
+                const uint32_t sb = smem_u32(b_parts) + combo[cidx][1] * kPartBytes;
 #pragma unroll
-        for (int b = 0; b < 4; ++b) {
-            int j = j0 + tx * 4 + b;
-            if (j < nb) out[j] = sm_scale * acc[a][b];
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                    umma_ss(tmem, make_smem_desc_sw128(sa + off, 16, 1024), make_smem_desc_sw128(sb + off, 16, 1024),
+                            idesc, first ? 0u : 1u);
+                    first = false;
+                }
+            }
+            umma_commit(smem_u32(&bar_done));
+        } else {
+            abort_flag = 1;
         }
+    }
+    ok = mbar_wait(smem_u32(&bar_done), 0, &abort_flag);
+    if (__syncthreads_and(ok ? 1 : 0)) {
+        tc_fence_after();
+        const int i = i0 + tid;                                    // this thread's row = its TMEM lane
+        float* out = scores + ((int64_t)bh * nb + i) * score_stride + j0;
+        const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+#pragma unroll
+        for (int ch = 0; ch < 4; ++ch) {
+            uint32_t r[32];
+            tmem_ld32(lane_addr + ch * 32, r);
+            tmem_wait_ld();
+            if (i < nb) {
+#pragma unroll
+                for (int c4 = 0; c4 < 32; c4 += 4) {
+                    if (j0 + ch * 32 + c4 < score_stride)           // score_stride is a multiple of 4
+                        *reinterpret_cast<float4*>(out + ch * 32 + c4) =
+                            make_float4(sm_scale * __uint_as_float(r[c4]), sm_scale * __uint_as_float(r[c4 + 1]),
+                                        sm_scale * __uint_as_float(r[c4 + 2]), sm_scale * __uint_as_float(r[c4 + 3]));
+                }
+            }
+        }
+    } else if (tid == 0) {
+        report_error(workspace, FVATTN_ERR_DEVICE_TIMEOUT, 0x9002u);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) {
+        tc_fence_after();
+        tmem_dealloc(tmem, 128);
     }
 }
 
@@ -313,15 +445,15 @@ select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int
     if (row >= n_rows) return;
     const float* srow = scores + row * score_stride;
 
-    float prob[E];
+    float sc[E];
     uint32_t key[E];
+    uint32_t mass_fx[E];   // probability in fixed point, 2^31 = 1: masses add exactly and warp-reduce in one instruction
     float mx = -INFINITY;
 #pragma unroll
     for (int e = 0; e < E; ++e) {
         const int j = lane + 32 * e;
-        const float sc = (j < nb) ? srow[j] + 0.0f : -INFINITY;   // -0 -> +0: equal scores, equal keys
-        prob[e] = sc;
-        mx = fmaxf(mx, sc);
+        sc[e] = (j < nb) ? srow[j] + 0.0f : -INFINITY;   // -0 -> +0: equal scores, equal keys
+        mx = fmaxf(mx, sc[e]);
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
@@ -329,61 +461,63 @@ select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int
 #pragma unroll
     for (int e = 0; e < E; ++e) {
         const int j = lane + 32 * e;
-        uint32_t u = __float_as_uint(prob[e]);
+        uint32_t u = __float_as_uint(sc[e]);
         u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-        key[e] = (j < nb) ? ~u : 0xffffffffu;                   // ascending key = descending score
-        const float ex = (j < nb) ? expf(prob[e] - mx) : 0.f;
-        prob[e] = ex;
-        z += ex;
+        key[e] = (j < nb) ? ~u : 0xffffffffu;            // ascending key = descending score
+        sc[e] = (j < nb) ? expf(sc[e] - mx) : 0.f;
+        z += sc[e];
     }
     z = warp_sum(z);
+    const float to_fx = 2147483648.0f / z;
 #pragma unroll
-    for (int e = 0; e < E; ++e) prob[e] = prob[e] / z;
+    for (int e = 0; e < E; ++e) mass_fx[e] = __float2uint_rn(sc[e] * to_fx);
 
     const int need_cnt = max(1, min(k_floor, nb));
+    const uint32_t p_fx = p > 0.f ? __float2uint_ru(p * 2147483648.0f) : 0u;
     uint32_t thr = 0xffffffffu;          // p >= 1 keeps everything
     int r_ties = 1 << 30;                // how many blocks with key == thr are kept (index order)
     if (p < 1.0f) {
-        uint32_t lo = 0u, hi = 0xffffffffu;
+        uint32_t lo = __reduce_min_sync(0xffffffffu, key[0]), hi = 0xffffffffu;   // key[0] holds blocks 0..31
+#pragma unroll
+        for (int e = 1; e < E; ++e) lo = min(lo, __reduce_min_sync(0xffffffffu, key[e]));
 #pragma unroll 1
         while (lo < hi) {
             const uint32_t mid = lo + ((hi - lo) >> 1);
-            float mass = 0.f;
+            uint32_t mass = 0u;
             int cnt = 0;
 #pragma unroll
             for (int e = 0; e < E; ++e) {
                 const bool in = key[e] <= mid;
-                mass += in ? prob[e] : 0.f;
+                mass += in ? mass_fx[e] : 0u;
                 cnt += in ? 1 : 0;
             }
-            mass = warp_sum(mass);
-            cnt = warp_sum(cnt);
-            if (mass >= p && cnt >= need_cnt) hi = mid; else lo = mid + 1;
+            mass = __reduce_add_sync(0xffffffffu, mass);
+            cnt = __reduce_add_sync(0xffffffffu, cnt);
+            if (mass >= p_fx && cnt >= need_cnt) hi = mid; else lo = mid + 1;
         }
         thr = hi;
         // blocks tied with the threshold score: admit them one by one, lowest index first
-        float mass_lt = 0.f, p_tie = 0.f;
+        uint32_t mass_lt = 0u, p_tie = 0u;
         int cnt_lt = 0, n_tie = 0;
 #pragma unroll
         for (int e = 0; e < E; ++e) {
             const bool lt = key[e] < thr, eq = key[e] == thr && (lane + 32 * e) < nb;
-            mass_lt += lt ? prob[e] : 0.f;
+            mass_lt += lt ? mass_fx[e] : 0u;
             cnt_lt += lt ? 1 : 0;
             n_tie += eq ? 1 : 0;
-            p_tie = eq ? prob[e] : p_tie;
+            p_tie = eq ? mass_fx[e] : p_tie;
         }
-        mass_lt = warp_sum(mass_lt);
-        cnt_lt = warp_sum(cnt_lt);
-        n_tie = warp_sum(n_tie);
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) p_tie = fmaxf(p_tie, __shfl_xor_sync(0xffffffffu, p_tie, o));
+        mass_lt = __reduce_add_sync(0xffffffffu, mass_lt);
+        cnt_lt = __reduce_add_sync(0xffffffffu, cnt_lt);
+        n_tie = __reduce_add_sync(0xffffffffu, n_tie);
+        p_tie = __reduce_max_sync(0xffffffffu, p_tie);
         if (n_tie > 1) {
-            float cum = mass_lt;
+            uint32_t cum = mass_lt;
             int r = 0;
             while (r < n_tie) {
                 cum += p_tie;
                 ++r;
-                if (cum >= p && cnt_lt + r >= need_cnt) break;
+                if (cum >= p_fx && cnt_lt + r >= need_cnt) break;
             }
             r_ties = r;
         }
@@ -439,31 +573,84 @@ head_load_kernel(const int32_t* __restrict__ counts, int nb, float* __restrict__
 }
 
 // ------------------------------------------------------------------------------------ launch
+// ---- host side ------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn route_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            (void)cudaGetLastError();
+    }
+    return fn;
+}
+
+// [3 * BH, nb, d] bf16 (the split means), box = 1 x 128 rows x 64 columns, 128-byte swizzle,
+// rows past nb read as zero.
+static bool make_split_map(CUtensorMap* map, const void* base, int d, int nb, int64_t BH) {
+    EncodeTiledFn fn = route_encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)d, (cuuint64_t)nb, (cuuint64_t)(3 * BH)};
+    cuuint64_t strides[2] = {(cuuint64_t)d * 2, (cuuint64_t)nb * d * 2};
+    cuuint32_t box[3] = {64, 128, 1};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int D>
+static fvattn_status_t launch_stages(const void* q_r, const void* k_r, int64_t BH, const GridDims& m, float sm_scale,
+                                     __nv_bfloat16* qsplit, __nv_bfloat16* ksplit, float* scores, int score_stride,
+                                     int sms, void* workspace, cudaStream_t s) {
+    {
+        const size_t block_bytes = (size_t)m.bs * D * 2;
+        const size_t smem = kPoolStages * block_bytes + 2 * sizeof(float) * kPoolThreads * 8 + 2 * (size_t)m.nb;
+        const int64_t items = 2 * BH * m.nb;
+        const unsigned grid = (unsigned)(items < sms ? items : sms);
+        FVATTN_CUDA_OK(cudaFuncSetAttribute(pool_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        pool_kernel<D><<<grid, kPoolThreads, smem, s>>>((const uint4*)q_r, (const uint4*)k_r, qsplit, ksplit, m, BH,
+                                                       workspace);
+        if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
+    }
+    CUtensorMap mq, mk;
+    if (!make_split_map(&mq, qsplit, D, m.nb, BH) || !make_split_map(&mk, ksplit, D, m.nb, BH)) return FVATTN_ERR_CUDA;
+    const size_t smem = 6 * (size_t)128 * D * 2;
+    FVATTN_CUDA_OK(cudaFuncSetAttribute(score_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    const unsigned tiles = (unsigned)((m.nb + 127) / 128);
+    score_tc_kernel<D><<<dim3(tiles, tiles, (unsigned)BH), sc::kThreads, smem, s>>>(mq, mk, scores, m.nb, (int)BH,
+                                                                                  score_stride, sm_scale, workspace);
+    return launch_status();
+}
+
 fvattn_status_t launch_route(const void* q_r, const void* k_r, int64_t BH, int d, const GridDims& m, float p,
                              int k_floor, float sm_scale, uint32_t* mask_bits, int32_t* counts, uint16_t* idx,
                              float* head_load, void* workspace, cudaStream_t s) {
     RouteWs w = route_ws(BH, m.nb, d);
     char* ws = static_cast<char*>(workspace);
-    float* qbar = reinterpret_cast<float*>(ws + w.qbar);
-    float* kbar = reinterpret_cast<float*>(ws + w.kbar);
+    __nv_bfloat16* qsplit = reinterpret_cast<__nv_bfloat16*>(ws + w.qsplit);
+    __nv_bfloat16* ksplit = reinterpret_cast<__nv_bfloat16*>(ws + w.ksplit);
     float* scores = reinterpret_cast<float*>(ws + w.scores);
+    int dev = 0, sms = 0;
+    FVATTN_CUDA_OK(cudaGetDevice(&dev));
+    FVATTN_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
 
-    dim3 pgrid((unsigned)m.nb, (unsigned)BH, 2);
-    if (d == 128)
-        pool_kernel<128><<<pgrid, kPoolThreads, 0, s>>>((const uint4*)q_r, (const uint4*)k_r, qbar, kbar, m);
-    else
-        pool_kernel<64><<<pgrid, kPoolThreads, 0, s>>>((const uint4*)q_r, (const uint4*)k_r, qbar, kbar, m);
-    if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
+    fvattn_status_t st = d == 128 ? launch_stages<128>(q_r, k_r, BH, m, sm_scale, qsplit, ksplit, scores, w.score_stride,
+                                                       sms, workspace, s)
+                                  : launch_stages<64>(q_r, k_r, BH, m, sm_scale, qsplit, ksplit, scores, w.score_stride,
+                                                      sms, workspace, s);
+    if (st != FVATTN_OK) return st;
 
-    unsigned tiles = (unsigned)((m.nb + kScoreTile - 1) / kScoreTile);
-    score_kernel<<<dim3(tiles, tiles, (unsigned)BH), 256, 0, s>>>(qbar, kbar, scores, m.nb, d, w.score_stride,
-                                                                   sm_scale);
-    if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
-
+    const int64_t n_rows = BH * m.nb;
     if (m.nb <= 1024) {
         const int e = (m.nb + 31) / 32;
-        const int64_t n_rows = BH * m.nb;
-        fvattn_status_t st;
 #define FVATTN_SEL_CASE(E_) \
     if (e <= E_) st = launch_select_warp<E_>(scores, m.nb, n_rows, w.score_stride, p, k_floor, mask_bits, counts, idx, s); else
         FVATTN_SEL_CASE(1) FVATTN_SEL_CASE(4) FVATTN_SEL_CASE(8) FVATTN_SEL_CASE(12) FVATTN_SEL_CASE(16)
@@ -474,10 +661,10 @@ fvattn_status_t launch_route(const void* q_r, const void* k_r, int64_t BH, int d
     } else {
         int n2 = 2048;
         while (n2 < m.nb) n2 <<= 1;
-        size_t smem = (size_t)n2 * (8 + 4 + 4) + 2 * sizeof(uint32_t) * (size_t)(n2 / 32);
+        const size_t smem = (size_t)n2 * (8 + 4 + 4) + 2 * sizeof(uint32_t) * (size_t)(n2 / 32);
         FVATTN_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        select_kernel<<<(unsigned)(BH * m.nb), kSelThreads, smem, s>>>(scores, m.nb, n2, w.score_stride, p, k_floor,
-                                                                      mask_bits, counts, idx);
+        select_kernel<<<(unsigned)n_rows, kSelThreads, smem, s>>>(scores, m.nb, n2, w.score_stride, p, k_floor,
+                                                                 mask_bits, counts, idx);
         if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
     }
 
