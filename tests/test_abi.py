@@ -41,9 +41,10 @@ def test_workspace_bytes_and_shape_errors():
     g = fv.Grid(21, 45, 80, 1, 8, 16)
     n = fv.workspace_bytes(g, 1, 40, 128)
     nb = 630
-    # header + two pooled-mean tensors + the score matrix (row stride rounded to 4 floats)
-    assert n >= 256 + 2 * 40 * nb * 128 * 4 + 40 * nb * 632 * 4
-    assert n < 256 + 2 * 40 * nb * 128 * 4 + 40 * nb * 632 * 4 + 4096
+    # header + pooled means of Q and K as three bf16 parts each + the score matrix (row stride
+    # rounded to 4 floats)
+    want = 256 + 2 * 3 * 40 * nb * 128 * 2 + 40 * nb * 632 * 4
+    assert want <= n < want + 4096
     with pytest.raises(fv.FvattnError) as e:
         fv.workspace_bytes(g, 1, 40, 96)                      # d not in {64, 128}
     assert e.value.status == fv.ERR_UNSUPPORTED_SHAPE
