@@ -21,8 +21,12 @@ namespace fvattn {
 using namespace ptx;
 
 // ------------------------------------------------------------------------------------ pool
+// Two CTAs per SM, each with a two-stage ring: while one CTA adds a block up, the other's copy
+// is in flight, which measured at the copy bandwidth of the device (one CTA with a four-stage
+// ring was 25 % slower: its single barrier per block serialised copy-wait and reduction).
 constexpr int kPoolThreads = 256;
-constexpr int kPoolStages = 4;
+constexpr int kPoolStages = 2;
+constexpr int kPoolCtasPerSm = 2;
 
 // x = hi + mid + lo exactly (3 x 8 significant bits), each part a bf16.
 __device__ __forceinline__ void split3(float x, __nv_bfloat16& hi, __nv_bfloat16& mid, __nv_bfloat16& lo) {
@@ -33,7 +37,7 @@ __device__ __forceinline__ void split3(float x, __nv_bfloat16& hi, __nv_bfloat16
 }
 
 template <int D>
-__global__ void __launch_bounds__(kPoolThreads)
+__global__ void __launch_bounds__(kPoolThreads, kPoolCtasPerSm)
 pool_kernel(const uint4* __restrict__ q_r, const uint4* __restrict__ k_r, __nv_bfloat16* __restrict__ qsplit,
             __nv_bfloat16* __restrict__ ksplit, GridDims m, int64_t BH, void* workspace) {
     constexpr int VPR = D / 8;                // 16-byte vectors per row
@@ -416,10 +420,11 @@ select_kernel(const float* __restrict__ scores, int nb, int n2, int score_stride
 }
 
 // One warp per (head, query block) row, nb <= 1024: the row lives in registers (E = ceil(nb/32)
-// entries per lane, block j = lane + 32 e).  Instead of sorting, the warp bisects on the 32-bit
-// order-preserving image of the score: the smallest threshold t such that the blocks with
-// key <= t hold mass >= p and number at least max(1, min(k_floor, nb)) is the key of the last
-// kept block, so {key <= t} is exactly the prefix the descending sort would have kept.  Blocks
+// entries per lane, block j = lane + 32 e).  Instead of sorting, the warp finds the key of the last
+// kept block by radix selection on the 32-bit order-preserving image of the score (ascending key =
+// descending score): the smallest key t such that the blocks with key <= t hold mass >= p and
+// number at least max(1, min(k_floor, nb)); {key <= t} is exactly the prefix a descending sort
+// would have kept.  Masses are fixed point (2^31 = 1) so they add exactly in any order.  Blocks
 // whose score equals the threshold's are admitted in index order one at a time (the tie rule).
 // The ballot of the keep flags over entry e is the mask word for blocks 32e..32e+31, and its
 // prefix pop-counts give the ascending compact index list.
@@ -440,6 +445,7 @@ template <int E>
 __global__ void __launch_bounds__(kSelWarpsPerCta * 32)
 select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int score_stride, float p, int k_floor,
                    uint32_t* __restrict__ mask_bits, int32_t* __restrict__ counts, uint16_t* __restrict__ idx) {
+    __shared__ uint32_t hist[kSelWarpsPerCta * 512];
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * kSelWarpsPerCta + (threadIdx.x >> 5);
     if (row >= n_rows) return;
@@ -457,13 +463,20 @@ select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+    float mn = INFINITY;
+#pragma unroll
+    for (int e = 0; e < E; ++e) mn = fminf(mn, (lane + 32 * e) < nb ? sc[e] : INFINITY);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) mn = fminf(mn, __shfl_xor_sync(0xffffffffu, mn, o));
+    // Selection key: distance below the row maximum on a linear 28-bit scale (ascending key =
+    // descending score).  The map is monotone; scores closer than range / 2^28 (below one fp32 ulp
+    // of the scores that matter) share a key and are then ordered by block index.
+    const float key_scale = (mx > mn) ? 268435200.0f / (mx - mn) : 0.f;
     float z = 0.f;
 #pragma unroll
     for (int e = 0; e < E; ++e) {
         const int j = lane + 32 * e;
-        uint32_t u = __float_as_uint(sc[e]);
-        u = (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-        key[e] = (j < nb) ? ~u : 0xffffffffu;            // ascending key = descending score
+        key[e] = (j < nb) ? min(__float2uint_rn((mx - sc[e]) * key_scale), 268435455u) : 0xffffffffu;
         sc[e] = (j < nb) ? expf(sc[e] - mx) : 0.f;
         z += sc[e];
     }
@@ -477,47 +490,113 @@ select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int
     uint32_t thr = 0xffffffffu;          // p >= 1 keeps everything
     int r_ties = 1 << 30;                // how many blocks with key == thr are kept (index order)
     if (p < 1.0f) {
-        uint32_t lo = __reduce_min_sync(0xffffffffu, key[0]), hi = 0xffffffffu;   // key[0] holds blocks 0..31
-#pragma unroll
-        for (int e = 1; e < E; ++e) lo = min(lo, __reduce_min_sync(0xffffffffu, key[e]));
-#pragma unroll 1
-        while (lo < hi) {
-            const uint32_t mid = lo + ((hi - lo) >> 1);
-            uint32_t mass = 0u;
-            int cnt = 0;
-#pragma unroll
-            for (int e = 0; e < E; ++e) {
-                const bool in = key[e] <= mid;
-                mass += in ? mass_fx[e] : 0u;
-                cnt += in ? 1 : 0;
-            }
-            mass = __reduce_add_sync(0xffffffffu, mass);
-            cnt = __reduce_add_sync(0xffffffffu, cnt);
-            if (mass >= p_fx && cnt >= need_cnt) hi = mid; else lo = mid + 1;
-        }
-        thr = hi;
-        // blocks tied with the threshold score: admit them one by one, lowest index first
-        uint32_t mass_lt = 0u, p_tie = 0u;
-        int cnt_lt = 0, n_tie = 0;
+        // Radix selection of the boundary key, 8 bits per pass, over the bits in which the row's keys
+        // differ: per pass a 256-bin histogram of (count, mass) of the keys that match the decided
+        // prefix, then a scan for the first bin where the running (mass, count) meets (p, floor).
+        uint32_t* hm = hist + (threadIdx.x >> 5) * 512;   // masses
+        uint32_t* hc = hm + 256;                          // counts
+        uint32_t kmin = 0xffffffffu, kmax = 0u;
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            const bool lt = key[e] < thr, eq = key[e] == thr && (lane + 32 * e) < nb;
-            mass_lt += lt ? mass_fx[e] : 0u;
-            cnt_lt += lt ? 1 : 0;
+            const bool real = (lane + 32 * e) < nb;
+            kmin = min(kmin, key[e]);
+            kmax = max(kmax, real ? key[e] : 0u);
+        }
+        kmin = __reduce_min_sync(0xffffffffu, kmin);
+        kmax = __reduce_max_sync(0xffffffffu, kmax);
+        int shift = 32 - __clz(kmin ^ kmax);              // keys agree on bits [shift, 32)
+        uint32_t prefix = shift >= 32 ? 0u : (kmin >> shift) << shift;
+        uint32_t mass_acc = 0u, cnt_acc = 0u;
+        bool reached = true;
+#pragma unroll 1
+        while (shift > 0 && reached) {
+            const int w = min(8, shift);
+            const int hi_shift = shift;                   // bits [hi_shift, 32) are decided
+            shift -= w;
+            const uint32_t bin_mask = (1u << w) - 1u;
+#pragma unroll
+            for (int t = 0; t < 16; ++t) hm[lane + 32 * t] = 0u;   // clears hm and hc (512 words)
+            __syncwarp();
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const bool match = (key[e] >> hi_shift) == (prefix >> hi_shift);   // pads (0xffffffff) never match
+                if (match) {
+                    const uint32_t bin = (key[e] >> shift) & bin_mask;
+                    atomicAdd(&hm[bin], mass_fx[e]);
+                    atomicAdd(&hc[bin], 1u);
+                }
+            }
+            __syncwarp();
+            // lane l owns bins 8l .. 8l+7
+            uint32_t bm[8], bc[8], tm = 0u, tcn = 0u;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                bm[t] = hm[8 * lane + t];
+                bc[t] = hc[8 * lane + t];
+                tm += bm[t];
+                tcn += bc[t];
+            }
+            uint32_t im = tm, ic = tcn;                   // inclusive scan over lanes
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t nm = __shfl_up_sync(0xffffffffu, im, o), nc = __shfl_up_sync(0xffffffffu, ic, o);
+                if (lane >= o) { im += nm; ic += nc; }
+            }
+            uint32_t run_m = mass_acc + im - tm, run_c = cnt_acc + ic - tcn;   // before this lane's bins
+            int local = 8;
+            uint32_t before_m = 0u, before_c = 0u, in_bin = 0u;
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                const uint32_t nm = run_m + bm[t], nc = run_c + bc[t];
+                if (local == 8 && nm >= p_fx && nc >= (uint32_t)need_cnt) {
+                    local = t;
+                    before_m = run_m;
+                    before_c = run_c;
+                    in_bin = bc[t];
+                }
+                run_m = nm;
+                run_c = nc;
+            }
+            const uint32_t found = __ballot_sync(0xffffffffu, local < 8);
+            if (found == 0u) {
+                reached = false;                           // the whole row holds less than p: keep everything
+            } else {
+                const int src = __ffs(found) - 1;
+                const uint32_t b = 8u * src + (uint32_t)__shfl_sync(0xffffffffu, local, src);
+                mass_acc = __shfl_sync(0xffffffffu, before_m, src);
+                cnt_acc = __shfl_sync(0xffffffffu, before_c, src);
+                prefix |= b << shift;
+                if (__shfl_sync(0xffffffffu, in_bin, src) == 1u && shift > 0) {
+                    // a single block is left in the chosen bin: its key is the threshold
+                    uint32_t cand = 0xffffffffu;
+#pragma unroll
+                    for (int e = 0; e < E; ++e)
+                        if ((key[e] >> shift) == (prefix >> shift)) cand = key[e];
+                    prefix = __reduce_min_sync(0xffffffffu, cand);
+                    shift = 0;
+                }
+            }
+            __syncwarp();
+        }
+        thr = reached ? prefix : kmax;
+        // blocks tied with the threshold score: admit them one by one, lowest index first
+        uint32_t p_tie = 0u;
+        int n_tie = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const bool eq = key[e] == thr && (lane + 32 * e) < nb;
             n_tie += eq ? 1 : 0;
             p_tie = eq ? mass_fx[e] : p_tie;
         }
-        mass_lt = __reduce_add_sync(0xffffffffu, mass_lt);
-        cnt_lt = __reduce_add_sync(0xffffffffu, cnt_lt);
         n_tie = __reduce_add_sync(0xffffffffu, n_tie);
-        p_tie = __reduce_max_sync(0xffffffffu, p_tie);
-        if (n_tie > 1) {
-            uint32_t cum = mass_lt;
+        if (n_tie > 1 && reached) {
+            p_tie = __reduce_max_sync(0xffffffffu, p_tie);
+            uint32_t cum = mass_acc;
             int r = 0;
             while (r < n_tie) {
                 cum += p_tie;
                 ++r;
-                if (cum >= p_fx && cnt_lt + r >= need_cnt) break;
+                if (cum >= p_fx && (int)cnt_acc + r >= need_cnt) break;
             }
             r_ties = r;
         }
@@ -614,7 +693,7 @@ static fvattn_status_t launch_stages(const void* q_r, const void* k_r, int64_t B
         const size_t block_bytes = (size_t)m.bs * D * 2;
         const size_t smem = kPoolStages * block_bytes + 2 * sizeof(float) * kPoolThreads * 8 + 2 * (size_t)m.nb;
         const int64_t items = 2 * BH * m.nb;
-        const unsigned grid = (unsigned)(items < sms ? items : sms);
+        const unsigned grid = (unsigned)(items < sms * kPoolCtasPerSm ? items : sms * kPoolCtasPerSm);
         FVATTN_CUDA_OK(cudaFuncSetAttribute(pool_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         pool_kernel<D><<<grid, kPoolThreads, smem, s>>>((const uint4*)q_r, (const uint4*)k_r, qsplit, ksplit, m, BH,
                                                        workspace);
