@@ -93,13 +93,6 @@ class ClockSampler:
                 "samples": len(sm)}
 
 
-def dist_env():
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    return rank, world, local
-
-
 def time_steps(fn, steps, torch):
     """CUDA-event time of `steps` calls of fn on the current stream, in ms (total)."""
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -164,10 +157,12 @@ def oracle_sample(cfg, budget_s, n_tiles_cap=64):
 
 def run_reference(args):
     """`--impl reference`: the CPU oracle as it stands, on the host cores, same metric and config."""
+    from paper_2607_16190_b200 import synth
+    from paper_2607_16190_b200.replicas import dist_env
+
     rank, world, _ = dist_env()
     if rank != 0:
         return
-    from paper_2607_16190_b200 import synth
 
     cfg = synth.CONFIGS[args.workload]
     per_step_budget = max(2.0, min(20.0, 150.0 / max(1, args.steps + args.warmup)))
@@ -206,9 +201,9 @@ def run_ours(args):
     import torch.distributed as dist
 
     from paper_2607_16190_b200 import binding as fv
-    from paper_2607_16190_b200 import synth
+    from paper_2607_16190_b200 import replicas, synth
 
-    rank, world, local = dist_env()
+    rank, world, local = replicas.dist_env()
     if world != args.gpus:
         raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}: launch with torch.distributed.run")
     torch.cuda.set_device(local)
@@ -217,7 +212,7 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=dev)
     fv.lib()                                                      # fail loudly if the extension is missing
 
-    cfg = synth.CONFIGS[args.workload].with_(seed=synth.CONFIGS[args.workload].seed + 100 * rank)
+    cfg = synth.CONFIGS[args.workload].with_(seed=replicas.replica_seed(synth.CONFIGS[args.workload].seed, rank))
     g = fv.Grid(*cfg.grid, *cfg.tile)
     nb = g.num_blocks
     q, k, v, _ = synth.make_qkv(cfg, dev)
@@ -271,15 +266,8 @@ def run_ours(args):
     for ev in events:
         for n, (a, b) in zip(stage_names, zip(ev[:-1], ev[1:])):
             stage_ms[n] += a.elapsed_time(b) / args.steps
-    if world > 1:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-        fl = torch.tensor([float(flops)], device=dev, dtype=torch.float64)
-        dist.all_reduce(fl, op=dist.ReduceOp.SUM)
-        flops_all = float(fl.item())
-    else:
-        flops_all = float(flops)
+    rate, total_ms = replicas.job_throughput(float(flops), total_ms, world, dev)
+    flops_all = rate * total_ms * 1e-3
     ms_per_step = total_ms / args.steps
     value = flops_all / (ms_per_step * 1e-3) / 1e12
 
@@ -298,10 +286,7 @@ def run_ours(args):
         dist.barrier()
     e2e_steps = max(2, min(args.steps, 5))
     e2e_ms = time_steps(e2e_step, e2e_steps, torch) / e2e_steps
-    if world > 1:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+    e2e_ms = replicas.max_over_ranks(e2e_ms, world, dev)
     e2e = {"value": flops_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
            "h2d_bytes_per_step": 3 * hq.numel() * 2, "d2h_bytes_per_step": hout.numel() * 2}
     del hq, hk, hv, hout, dq, dk, dv
