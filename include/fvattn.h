@@ -133,6 +133,39 @@ fvattn_status_t fvattn_sparse_attn_simt(const void* q_r, const void* k_r, const 
                                         const fvattn_grid_t* grid, float sm_scale, void* o_r, void* workspace,
                                         size_t workspace_bytes, fvattn_stream_t stream);
 
+/*
+ * fvattn_sparse_attn without a workspace and without any allocation.  (The paper has no
+ * counterpart to this call: it exists for the way this library is embedded, not for the method.)
+ *
+ * Who needs it: hosts that gave all of the device's memory to their own arena when they started
+ * (a serving process, an engine plug-in), so that a later cudaMalloc fails or is forbidden by
+ * their rules, and code on a latency-critical path that must not pay cudaMalloc's device-wide
+ * synchronisation.  Such a caller may have nowhere to take the workspace of fvattn_sparse_attn
+ * from.  Here the scratch (tile order, key-validity table, per-head totals, tile counter, error
+ * word) is a fixed 1 MiB array in the library's own device image: every GPU on which the
+ * library is used holds that 1 MiB from the time its image is loaded there until the process
+ * exits.  The call itself never calls cudaMalloc, cudaFree or any routine that allocates.
+ *
+ * Same inputs, output and arithmetic as fvattn_sparse_attn.  Differences:
+ *   - shapes whose scratch would exceed the array (about B*H*nb > 240,000 tiles) are rejected
+ *     with FVATTN_ERR_WORKSPACE_TOO_SMALL before anything is launched;
+ *   - the array is shared by every call on that GPU and keeps the previous call's contents; the
+ *     call clears the part that must start at zero on `stream` before its kernels.  Two calls
+ *     that overlap on the GPU (different streams, or different host threads without ordering)
+ *     race on it: order them on one stream or with events;
+ *   - the first call on a device looks up the array's device address (once per device, with
+ *     that device current).  Make that first call outside any stream capture;
+ *   - status_out (device pointer to two uint32, may be NULL): receives the error word and its
+ *     detail at the end of the call, in stream order (0 = no device-side error; otherwise
+ *     FVATTN_ERR_DEVICE_TIMEOUT or FVATTN_ERR_DEVICE_BOUNDS), since there is no caller
+ *     workspace for fvattn_device_status to read.
+ */
+fvattn_status_t fvattn_sparse_attn_noalloc(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
+                                           const int32_t* counts, int32_t B, int32_t H, int32_t d,
+                                           const fvattn_grid_t* grid, float sm_scale, void* o_r,
+                                           uint32_t* status_out /* device, 2 words, may be NULL */,
+                                           fvattn_stream_t stream);
+
 /* The heaviest-first tile order fvattn_sparse_attn builds from `counts` (Sec. 2.2's
  * observation that per-head workloads differ, applied inside one GPU): order[t] = bh*nb + i.
  * Exported for inspection and tests.  order: u32 [B*H*nb]. */

@@ -23,7 +23,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, E
 EXPORTS = (
     "fvattn_num_blocks", "fvattn_block_tokens", "fvattn_padded_tokens", "fvattn_workspace_bytes",
     "fvattn_workspace_init", "fvattn_reorder", "fvattn_inverse_reorder", "fvattn_route",
-    "fvattn_sparse_attn", "fvattn_sparse_attn_simt", "fvattn_tile_order", "fvattn_device_status",
+    "fvattn_sparse_attn", "fvattn_sparse_attn_simt", "fvattn_sparse_attn_noalloc", "fvattn_tile_order", "fvattn_device_status",
     "fvattn_status_string",
 )
 
@@ -231,6 +231,23 @@ def sparse_attn_simt(q_r, k_r, v_r, idx, counts, grid: Grid, sm_scale: float | N
                      out: torch.Tensor | None = None) -> torch.Tensor:
     """Same contract on the CUDA-core kernel (cross-check; the path for Bs or d = 64)."""
     return _attn("fvattn_sparse_attn_simt", q_r, k_r, v_r, idx, counts, grid, sm_scale, workspace, out)
+
+
+def sparse_attn_noalloc(q_r, k_r, v_r, idx, counts, grid: Grid, sm_scale: float | None, out: torch.Tensor,
+                        status_out: torch.Tensor | None = None) -> torch.Tensor:
+    """fvattn_sparse_attn for callers that cannot allocate: no workspace argument (the scratch is a
+    fixed array inside the library) and `out` must be supplied, so nothing is allocated anywhere on
+    the way.  `status_out` (2 x uint32 on the device, optional) receives the device error word."""
+    _need_cuda(q_r, k_r, v_r, idx, counts, out)
+    B, H, n_pad, d = q_r.shape
+    assert all(t.is_contiguous() for t in (q_r, k_r, v_r, idx, counts, out))
+    assert idx.dtype == torch.uint16 and counts.dtype == torch.int32
+    if sm_scale is None:
+        sm_scale = 1.0 / math.sqrt(d)
+    _check(lib().fvattn_sparse_attn_noalloc(_ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(idx), _ptr(counts), B, H, d,
+                                            ctypes.byref(grid.c()), ctypes.c_float(sm_scale), _ptr(out),
+                                            _ptr(status_out), _stream()), "fvattn_sparse_attn_noalloc")
+    return out
 
 
 def tile_order(counts: torch.Tensor, grid: Grid, workspace: torch.Tensor) -> torch.Tensor:

@@ -1,0 +1,79 @@
+// fvattn_sparse_attn_noalloc: block-sparse attention for callers that cannot hand the library a
+// workspace.  The scratch the attention path needs (the heaviest-first tile order, the per-block
+// key-validity table, the per-head totals and the header with the tile counter and the error
+// word) lives in a fixed array in device global memory that is part of this library's image, so
+// the call needs no buffer from the caller and allocates nothing.
+#include <mutex>
+
+#include "common.cuh"
+
+namespace fvattn {
+
+// Upper bound of the scratch, fixed at build time.  Every GPU on which the library is used holds
+// this much device memory from the moment the library's image is loaded there until the process
+// exits.
+constexpr size_t kStaticScratchBytes = 1u << 20;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// In host code `g_static_scratch` is only a handle for the runtime, not an address a kernel can
+// use: the device address is looked up once per device with cudaGetSymbolAddress and cached.
+static void* g_scratch_addr[64];
+static bool g_scratch_known[64];
+static std::mutex g_scratch_mutex;
+
+static fvattn_status_t static_scratch(void** out) {
+    int dev = -1;
+    FVATTN_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return FVATTN_ERR_CUDA;
+    std::lock_guard<std::mutex> lock(g_scratch_mutex);
+    if (!g_scratch_known[dev]) {
+        void* ptr = nullptr;
+        FVATTN_CUDA_OK(cudaGetSymbolAddress(&ptr, g_static_scratch));   // for the current device
+        g_scratch_addr[dev] = ptr;
+        g_scratch_known[dev] = true;
+    }
+    *out = g_scratch_addr[dev];
+    return FVATTN_OK;
+}
+
+} // namespace fvattn
+
+using namespace fvattn;
+
+extern "C" fvattn_status_t fvattn_sparse_attn_noalloc(const void* q_r, const void* k_r, const void* v_r,
+                                                      const uint16_t* idx, const int32_t* counts, int32_t B,
+                                                      int32_t H, int32_t d, const fvattn_grid_t* grid,
+                                                      float sm_scale, void* o_r, uint32_t* status_out,
+                                                      fvattn_stream_t stream) {
+    if (!q_r || !k_r || !v_r || !idx || !counts || !o_r || !grid_ok(grid)) return FVATTN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || !(sm_scale > 0.f) || isinf(sm_scale)) return FVATTN_ERR_INVALID_ARG;
+    const GridDims m = make_dims(*grid);
+    if (!((d == 64 || d == 128) && (m.bs == 64 || m.bs == 128) && m.nb >= 1 && m.nb <= kMaxBlocks))
+        return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    const int64_t BH = (int64_t)B * H;
+    if (BH * m.nb > 0x7fffffffLL) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(q_r, 128) || !aligned(k_r, 128) || !aligned(v_r, 128) || !aligned(o_r, 128) || !aligned(idx, 2) ||
+        !aligned(counts, 4) || (status_out && !aligned(status_out, 4)))
+        return FVATTN_ERR_INVALID_ARG;
+    const AttnWs w = attn_ws(BH, m.nb);
+    if (w.total > kStaticScratchBytes) return FVATTN_ERR_WORKSPACE_TOO_SMALL;   // shape beyond the fixed scratch
+
+    void* scratch = nullptr;
+    fvattn_status_t st = static_scratch(&scratch);
+    if (st != FVATTN_OK) return st;
+    cudaStream_t s = (cudaStream_t)stream;
+    // the array keeps what the previous call left: the header (error word, tile counter) must start at zero
+    FVATTN_CUDA_OK(cudaMemsetAsync(scratch, 0, kWsHeaderBytes, s));
+    uint32_t* order = reinterpret_cast<uint32_t*>(static_cast<char*>(scratch) + w.order);
+    st = launch_tile_order(counts, BH, m.nb, order, scratch, s);
+    if (st != FVATTN_OK) return st;
+    if (m.bs == 128 && d == 128)
+        st = launch_attn_tc(q_r, k_r, v_r, idx, counts, BH, m, sm_scale, o_r, order, scratch, s);
+    else
+        st = launch_attn_simt(q_r, k_r, v_r, idx, counts, BH, d, m, sm_scale, o_r, order, scratch, s);
+    if (st != FVATTN_OK) return st;
+    if (status_out)
+        FVATTN_CUDA_OK(cudaMemcpyAsync(status_out, scratch, 2 * sizeof(uint32_t), cudaMemcpyDeviceToDevice, s));
+    return FVATTN_OK;
+}
