@@ -65,6 +65,27 @@ __device__ __forceinline__ float ex2(float x) {
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+// (x, y) <- (x, y) * a + b, one packed fp32x2 instruction
+__device__ __forceinline__ void fma2(float& x, float& y, float a, float b) {
+    unsigned long long v, va, vb;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(v) : "f"(x), "f"(y));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(va) : "f"(a));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(vb) : "f"(b));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(v) : "l"(v), "l"(va), "l"(vb));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(x), "=f"(y) : "l"(v));
+}
+// acc + (bf16 in the low / high half of a packed pair), fp32 result
+__device__ __forceinline__ void add_bf16_pair(float& acc_lo, float& acc_hi, uint32_t packed) {
+    unsigned short lo, hi;
+    asm("mov.b32 {%0, %1}, %2;" : "=h"(lo), "=h"(hi) : "r"(packed));
+    asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(acc_lo) : "h"(lo));
+    asm("add.rn.f32.bf16 %0, %1, %0;" : "+f"(acc_hi) : "h"(hi));
+}
 template <int N>
 __device__ __forceinline__ void setmaxnreg_inc() {
     asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N));
@@ -327,11 +348,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 float mx0 = __uint_as_float(s[0]), mx1 = __uint_as_float(s[1]), mx2 = __uint_as_float(s[2]),
                       mx3 = __uint_as_float(s[3]);
 #pragma unroll
-                for (int j = 4; j < 128; j += 4) {
-                    mx0 = fmaxf(mx0, __uint_as_float(s[j]));
-                    mx1 = fmaxf(mx1, __uint_as_float(s[j + 1]));
-                    mx2 = fmaxf(mx2, __uint_as_float(s[j + 2]));
-                    mx3 = fmaxf(mx3, __uint_as_float(s[j + 3]));
+                for (int j = 4; j < 128; j += 8) {
+                    mx0 = max3(mx0, __uint_as_float(s[j]), __uint_as_float(s[j + 1]));
+                    mx1 = max3(mx1, __uint_as_float(s[j + 2]), __uint_as_float(s[j + 3]));
+                    if (j + 4 < 128) {
+                        mx2 = max3(mx2, __uint_as_float(s[j + 4]), __uint_as_float(s[j + 5]));
+                        mx3 = max3(mx3, __uint_as_float(s[j + 6]), __uint_as_float(s[j + 7]));
+                    }
                 }
                 const float m_new = fmaxf(m_run, fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3)));
                 // lazy rescale: keep the old reference max unless the new one is more than 2^8 above it
@@ -360,21 +383,19 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 uint32_t pk[64];
 #pragma unroll
                 for (int j = 0; j < 128; j += 4) {
-                    const float p0 = ex2(fmaf(__uint_as_float(s[j]), sl2, -moff));
-                    const float p1 = ex2(fmaf(__uint_as_float(s[j + 1]), sl2, -moff));
-                    const float p2 = ex2(fmaf(__uint_as_float(s[j + 2]), sl2, -moff));
-                    const float p3 = ex2(fmaf(__uint_as_float(s[j + 3]), sl2, -moff));
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(p0, p1);   // .x (low half) = even column
-                    __nv_bfloat162 hi = __floats2bfloat162_rn(p2, p3);
+                    float e0 = __uint_as_float(s[j]), e1 = __uint_as_float(s[j + 1]), e2 = __uint_as_float(s[j + 2]),
+                          e3 = __uint_as_float(s[j + 3]);
+                    fma2(e0, e1, sl2, -moff);
+                    fma2(e2, e3, sl2, -moff);
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(ex2(e0), ex2(e1));   // .x (low half) = even column
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(ex2(e2), ex2(e3));
                     const uint32_t wlo = *reinterpret_cast<uint32_t*>(&lo), whi = *reinterpret_cast<uint32_t*>(&hi);
                     pk[j >> 1] = wlo;
                     pk[(j >> 1) + 1] = whi;
                     // the row sum takes the bf16-rounded weights the second MMA sees, so numerator and
                     // denominator stay consistent (an exact weighted average of V)
-                    sum0 += __uint_as_float(wlo << 16);
-                    sum1 += __uint_as_float(wlo & 0xffff0000u);
-                    sum2 += __uint_as_float(whi << 16);
-                    sum3 += __uint_as_float(whi & 0xffff0000u);
+                    add_bf16_pair(sum0, sum1, wlo);
+                    add_bf16_pair(sum2, sum3, whi);
                 }
                 l_run += (sum0 + sum1) + (sum2 + sum3);
                 tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
