@@ -3,7 +3,8 @@
 //
 // One persistent CTA per SM, 12 warps, warp-specialised:
 //   warp 0        producer: pops (head, query-block) tiles from the heaviest-first queue, TMA-loads
-//                 Q once per tile and the retained K / V tiles by index into 3-deep rings
+//                 Q once per tile and the retained K tiles by index into a 3-deep ring
+//   warp 2        second producer: the retained V tiles into their own 3-deep ring
 //   warp 1        MMA issuer (one thread): S = Q K^T and O += P V as tcgen05 MMAs, accumulators in
 //                 tensor memory
 //   warps 4-7     softmax of the even retained blocks  (stream 0)
@@ -133,7 +134,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         mbar_init(smem_u32(&sm.o_free), 8);
         mbar_init(smem_u32(&sm.ml_ready), 8);
         mbar_init(smem_u32(&sm.ml_done), 8);
-        for (int s = 0; s < TS; ++s) { mbar_init(smem_u32(&sm.tile_full[s]), 1); mbar_init(smem_u32(&sm.tile_empty[s]), 9); }
+        for (int s = 0; s < TS; ++s) { mbar_init(smem_u32(&sm.tile_full[s]), 1); mbar_init(smem_u32(&sm.tile_empty[s]), 10); }
         sm.abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_q);
@@ -154,8 +155,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     if (warp < 4) {
         setmaxnreg_dec<40>();
         if (warp == 0) {
-            // ======================= producer =======================================================
-            uint32_t n = 0, kn = 0, vn = 0, qn = 0;
+            // ======================= Q / K producer and tile queue ======================================
+            uint32_t n = 0, kn = 0, qn = 0;
             bool ok = true;
             while (ok) {
                 const uint32_t slot = n % TS;
@@ -204,15 +205,55 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                                 kb = 0;   // keep the pipeline consistent; the tile's result is undefined
                             }
                             const int krow = (int)(head_row0 + (int64_t)kb * BS);
-                            const uint32_t ks = kn % KS, vs = vn % VS;
+                            const uint32_t ks = kn % KS;
                             ok = mbar_wait(smem_u32(&sm.k_empty[ks]), ((kn / KS) & 1u) ^ 1u, abort_flag);
                             if (ok) {
                                 const uint32_t bar = smem_u32(&sm.k_full[ks]);
                                 mbar_expect_tx(bar, kTileBytes);
                                 tma_load_2d(smem_u32(sm.k[ks]), &map_k, 0, krow, bar);
                                 tma_load_2d(smem_u32(sm.k[ks]) + kHalfBytes, &map_k, 64, krow, bar);
-                                ok = mbar_wait(smem_u32(&sm.v_empty[vs]), ((vn / VS) & 1u) ^ 1u, abort_flag);
                             }
+                        }
+                        ++kn;
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                }
+            }
+            failed = !ok;
+        } else if (warp == 2) {
+            // ======================= V producer ========================================================
+            // A second producer warp, so that a K tile is fetched the moment its ring slot frees (after
+            // the QK MMA) instead of queueing behind the wait for a V slot (freed only after the PV MMA).
+            uint32_t n = 0, vn = 0;
+            bool ok = true;
+            while (ok) {
+                const uint32_t slot = n % TS;
+                int tile = -1, c = 0;
+                if (lane == 0) {
+                    ok = mbar_wait(smem_u32(&sm.tile_full[slot]), (n / TS) & 1u, abort_flag);
+                    if (ok) {
+                        tile = sm.tile_id[slot];
+                        c = sm.tile_cnt[slot];
+                        mbar_arrive(smem_u32(&sm.tile_empty[slot]));
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                tile = __shfl_sync(0xffffffffu, tile, 0);
+                c = __shfl_sync(0xffffffffu, c, 0);
+                ++n;
+                if (!ok || tile < 0) break;
+                const int64_t head_row0 = (int64_t)((uint32_t)tile / (uint32_t)m.nb) * m.n_pad;
+                const uint16_t* irow = idx + (int64_t)tile * m.nb;
+                for (int t0 = 0; t0 < c && ok; t0 += 32) {
+                    const int mine = (t0 + lane < c) ? (int)irow[t0 + lane] : 0;
+                    const int lim = min(32, c - t0);
+                    for (int tt = 0; tt < lim; ++tt) {
+                        int kb = __shfl_sync(0xffffffffu, mine, tt);
+                        if (lane == 0 && ok) {
+                            if (kb >= m.nb) kb = 0;   // reported by the K producer
+                            const int krow = (int)(head_row0 + (int64_t)kb * BS);
+                            const uint32_t vs = vn % VS;
+                            ok = mbar_wait(smem_u32(&sm.v_empty[vs]), ((vn / VS) & 1u) ^ 1u, abort_flag);
                             if (ok) {
                                 const uint32_t bar = smem_u32(&sm.v_full[vs]);
                                 mbar_expect_tx(bar, kTileBytes);
@@ -220,7 +261,6 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                                 tma_load_2d(smem_u32(sm.v[vs]) + kHalfBytes, &map_v, 64, krow, bar);
                             }
                         }
-                        ++kn;
                         ++vn;
                     }
                     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -233,7 +273,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, true);
             uint32_t n = 0, kn = 0, vn = 0, qn = 0, pn[2] = {0, 0};
             bool ok = true;
-            const uint32_t sq = smem_u32(sm.q);
+            // descriptor words that never change: high word (stride 1024 B, version, 128-byte swizzle);
+            // low word = (address >> 4) | (leading offset >> 4) << 16, advanced by adding (bytes >> 4)
+            const uint32_t desc_hi = (uint32_t)(make_smem_desc_sw128(0, 16, 1024) >> 32);
+            const uint32_t q_lo = (uint32_t)make_smem_desc_sw128(smem_u32(sm.q), 16, 1024);
+            const uint32_t k_lo0 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.k[0]), 16, 1024);
+            const uint32_t v_lo0 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.v[0]), kHalfBytes, 1024);
 
             auto issue_pv = [&](int u) {
                 const int b = u & 1;
@@ -244,11 +289,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 if (u == 0) ok = ok && mbar_wait(smem_u32(&sm.o_free), (qn & 1u) ^ 1u, abort_flag);
                 if (ok) {
                     tc_fence_after();
-                    const uint32_t sv = smem_u32(sm.v[vs]);
+                    const uint32_t vlo = v_lo0 + vs * (kTileBytes >> 4);
+                    const uint32_t tOb = tmem + kColO + 128u * b, tPb = tmem + kColS + 128u * b;
 #pragma unroll
                     for (int ks = 0; ks < BS / 16; ++ks)
-                        umma_ts(tmem + kColO + 128u * b, tmem + kColS + 128u * b + ks * 8,
-                                make_smem_desc_sw128(sv + (uint32_t)ks * 2048u, kHalfBytes, 1024), idesc_pv,
+                        umma_ts(tOb, tPb + ks * 8, ((uint64_t)desc_hi << 32) | (vlo + (uint32_t)ks * (2048u >> 4)), idesc_pv,
                                 (u >= 2 || ks > 0) ? 1u : 0u);
                     umma_commit(smem_u32(&sm.v_empty[vs]));
                 }
@@ -272,12 +317,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                     ok = mbar_wait(smem_u32(&sm.k_full[ks_]), (kn / KS) & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-                    const uint32_t sk = smem_u32(sm.k[ks_]);
+                    const uint32_t klo = k_lo0 + ks_ * (kTileBytes >> 4);
+                    const uint32_t tSa = tmem + kColS + 128u * a;
 #pragma unroll
                     for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                        umma_ss(tmem + kColS + 128u * a, make_smem_desc_sw128(sq + off, 16, 1024),
-                                make_smem_desc_sw128(sk + off, 16, 1024), idesc_qk, ks > 0 ? 1u : 0u);
+                        const uint32_t off16 = ((uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u) >> 4;
+                        umma_ss(tSa, ((uint64_t)desc_hi << 32) | (q_lo + off16), ((uint64_t)desc_hi << 32) | (klo + off16),
+                                idesc_qk, ks > 0 ? 1u : 0u);
                     }
                     umma_commit(smem_u32(&sm.k_empty[ks_]));
                     ++kn;
