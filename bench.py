@@ -30,9 +30,12 @@ if ROOT not in sys.path:
 FLOP_PER_PAIR = 4 * 128 * 128 * 128          # 4*d*Bq*Bk, d = Bq = Bk = 128
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 METRIC = "sparse-attn effective TFLOPS per attention layer (4*d*Bq*Bk FLOP per retained block pair / time)"
-# dram__bytes_read.sum + dram__bytes_write.sum of one attn_tc_kernel launch, from the ncu capture
-# summarised under profiles/; None until a capture of the current kernel exists.
-ATTN_DRAM_TRAFFIC_BYTES_PER_PAIR = None
+# dram__bytes_read.sum + dram__bytes_write.sum of one attn_tc_kernel launch from the ncu capture
+# summarised in profiles/attn_tc_kernel_wan480p.md: 1.292 GB + 0.422 GB at wan480p = 996 B per
+# (head, padded token).  DRAM traffic of this kernel follows the size of Q, K, V, O (each is moved
+# once; K/V re-reads are served by L2), not the number of retained pairs, so the 720p figure is
+# the 480p capture scaled by H * N_pad.
+ATTN_DRAM_BYTES_PER_HEAD_TOKEN = (1.291587e9 + 0.421784e9) / (40 * 43008)
 
 
 def load_peaks():
@@ -306,7 +309,8 @@ def run_ours(args):
         "bound": "tensor", "achieved": attn_tflops, "peak": peak_t, "unit": "TFLOP/s", "frac": attn_tflops / peak_t,
         "peak_kind": f"{peaks_kind} sustained bf16 (kernel timed inside a long step)",
         "frac_of_burst_peak": attn_tflops / float(peaks["bf16_tflops"]), "burst_peak": float(peaks["bf16_tflops"]),
-        "traffic": None if ATTN_DRAM_TRAFFIC_BYTES_PER_PAIR is None else ATTN_DRAM_TRAFFIC_BYTES_PER_PAIR * pairs,
+        "traffic": ATTN_DRAM_BYTES_PER_HEAD_TOKEN * cfg.H * g.padded_tokens,
+        "traffic_note": "ncu capture at wan480p scaled by H*N_pad (bytes); algorithmic minimum = 4 tensors once",
         "algorithmic_flop_per_launch": flops, "ms_per_launch": attn_ms,
     }
     route_bytes = 2 * cfg.H * cfg.tokens * cfg.d * 2 + layer.routing.mask_bits.numel() * 4 + cfg.H * nb * 4 + pairs * 2
@@ -369,6 +373,64 @@ def dense_baselines(fv, layer, cfg, g, q, k, v, sparse_attn_ms, torch):
     return out
 
 
+def run_sweep(args):
+    """Config 5: the 720p shapes over `--sweep-layers` layer seeds at p in SWEEP_P; per p: density,
+    ms per layer (route + attention), effective TFLOP/s of the attention kernel, speedup vs dense."""
+    import torch
+
+    from paper_2607_16190_b200 import binding as fv
+    from paper_2607_16190_b200 import synth
+
+    torch.cuda.set_device(0)
+    base = synth.CONFIGS["wan720p"]
+    g = fv.Grid(*base.grid, *base.tile)
+    nb = g.num_blocks
+    layer = fv.SparseAttentionLayer(g, 1, base.H, base.d, 0.9, base.k_floor, device="cuda:0")
+    full = None
+    acc = {p: {"density": [], "route_ms": [], "attn_ms": []} for p in synth.SWEEP_P}
+    dense_own, dense_sdpa = [], []
+    for li in range(args.sweep_layers):
+        cfg = synth.sweep_layer(li)
+        q, k, v, _ = synth.make_qkv(cfg, "cuda:0")
+        for src, dst in ((q, layer.q_r), (k, layer.k_r), (v, layer.v_r)):
+            fv.reorder(src, g, dst)
+        for p in synth.SWEEP_P:
+            def route():
+                fv.route(layer.q_r, layer.k_r, g, p, cfg.k_floor, layer.sm_scale, layer.workspace, layer.routing)
+
+            def attn():
+                fv.sparse_attn(layer.q_r, layer.k_r, layer.v_r, layer.routing.idx, layer.routing.counts, g,
+                               layer.sm_scale, layer.workspace, layer.o_r)
+            route(); attn()                                   # warm-up for this (layer, p)
+            acc[p]["route_ms"].append(time_steps(route, 1, torch))
+            acc[p]["attn_ms"].append(time_steps(attn, 1, torch))
+            acc[p]["density"].append(int(layer.routing.counts.sum().item()) / (cfg.H * nb * nb))
+        if li < args.sweep_dense_layers:                      # dense baselines on the same inputs
+            full = fv.route(layer.q_r, layer.k_r, g, 1.0, cfg.k_floor, layer.sm_scale, layer.workspace, full)
+            own = lambda: fv.sparse_attn(layer.q_r, layer.k_r, layer.v_r, full.idx, full.counts, g, layer.sm_scale,
+                                         layer.workspace, layer.o_r)
+            own()
+            dense_own.append(time_steps(own, 1, torch))
+            qt, kt, vt = (t.transpose(1, 2) for t in (q, k, v))
+            f = lambda: torch.nn.functional.scaled_dot_product_attention(qt, kt, vt)
+            f()
+            dense_sdpa.append(time_steps(f, 1, torch))
+        del q, k, v
+    status = fv.device_status(layer.workspace)
+    mean = lambda xs: sum(xs) / len(xs)
+    rows = []
+    for p in synth.SWEEP_P:
+        a = acc[p]
+        pairs = mean(a["density"]) * base.H * nb * nb
+        rows.append({"p": p, "density": mean(a["density"]), "route_ms": mean(a["route_ms"]), "attn_ms": mean(a["attn_ms"]),
+                     "attn_ms_min": min(a["attn_ms"]), "attn_ms_max": max(a["attn_ms"]),
+                     "attn_tflops": pairs * FLOP_PER_PAIR / mean(a["attn_ms"]) / 1e9,
+                     "speedup_vs_dense_own_kernel": mean(dense_own) / mean(a["attn_ms"]),
+                     "speedup_vs_dense_sdpa": mean(dense_sdpa) / mean(a["attn_ms"])})
+    print(json.dumps({"sweep": "wan720p x %d layers" % args.sweep_layers, "device_status": fv.status_string(status),
+                      "dense_own_kernel_ms": mean(dense_own), "dense_sdpa_ms": mean(dense_sdpa), "rows": rows}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -379,8 +441,13 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the dense baselines")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline-multi", action="store_true", help="also time the oracle when N > 1")
+    ap.add_argument("--sweep", action="store_true", help="run the 720p layer x p sweep instead of the timed step")
+    ap.add_argument("--sweep-layers", type=int, default=40)
+    ap.add_argument("--sweep-dense-layers", type=int, default=4)
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
