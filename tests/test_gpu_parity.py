@@ -152,6 +152,49 @@ def test_route_sweep_layers_all_p(layer):
     assert fv.device_status(ws) == fv.OK
 
 
+def test_route_more_than_1024_blocks_uses_the_sorting_kernel():
+    """nb = 1280 > 1024: the CTA-wide bitonic-sort selection path, d = 64, 64-token blocks."""
+    cfg = synth.Config("many_blocks", 2, 64, (5, 128, 128), (1, 8, 8), 0.9, 3, 16, "loguniform", seed=31)
+    g, og = grids(cfg)
+    assert g.num_blocks == 1280
+    q, k, _, _ = synth.make_qkv(cfg, "cuda")
+    q_r, k_r = fv.reorder(q, g), fv.reorder(k, g)
+    ws = fv.make_workspace(g, 1, cfg.H, cfg.d)
+    qb, kb = synth.bf16_bits(q_r)[0], synth.bf16_bits(k_r)[0]
+    for p in (0.9, 0.0):
+        res = fv.route(q_r, k_r, g, p, cfg.k_floor, cfg.sm_scale, ws)
+        assert fv.device_status(ws) == fv.OK
+        res_o = O.route(qb, kb, og, p, cfg.k_floor, cfg.sm_scale)
+        ndiff, nnear, ntie = compare_masks(res, res_o, p)
+        print(f"\n[nb=1280 p={p}] differing {ndiff}, near-threshold {nnear}, near-tie {ntie}, "
+              f"density {res_o.counts.mean() / 1280:.4f}")
+
+
+def test_batch_of_two_routes_and_attends_like_two_single_batches():
+    """B = 2: (batch, head) pairs are independent; results equal the per-batch calls bit for bit."""
+    cfg = synth.CONFIGS["small"]
+    g, og = grids(cfg)
+    qa, ka, va, _ = synth.make_qkv(cfg, "cuda")
+    qb_, kb_, vb_, _ = synth.make_qkv(cfg.with_(seed=77), "cuda")
+    q, k, v = (torch.cat(t, 0) for t in ((qa, qb_), (ka, kb_), (va, vb_)))
+    q_r, k_r, v_r = (fv.reorder(t, g) for t in (q, k, v))
+    ws = fv.make_workspace(g, 2, cfg.H, cfg.d)
+    res = fv.route(q_r, k_r, g, cfg.p, cfg.k_floor, cfg.sm_scale, ws)
+    o_r = fv.sparse_attn(q_r, k_r, v_r, res.idx, res.counts, g, cfg.sm_scale, ws)
+    assert fv.device_status(ws) == fv.OK
+    ws1 = fv.make_workspace(g, 1, cfg.H, cfg.d)
+    for b, (q1, k1, v1) in enumerate(((qa, ka, va), (qb_, kb_, vb_))):
+        q1r, k1r, v1r = (fv.reorder(t, g) for t in (q1, k1, v1))
+        assert torch.equal(q1r[0], q_r[b])
+        r1 = fv.route(q1r, k1r, g, cfg.p, cfg.k_floor, cfg.sm_scale, ws1)
+        assert torch.equal(r1.counts[0], res.counts[b])
+        assert torch.equal(r1.mask_bits.view(torch.int32)[0], res.mask_bits.view(torch.int32)[b])
+        o1 = fv.sparse_attn(q1r, k1r, v1r, r1.idx, r1.counts, g, cfg.sm_scale, ws1)
+        assert torch.equal(o1[0], o_r[b])
+    back = fv.inverse_reorder(o_r, g)
+    assert back.shape == q.shape
+
+
 # ------------------------------------------------------------------------------ tile order
 @pytest.mark.parametrize("name", ["small", "wan480p"])
 def test_tile_order_is_heaviest_first_permutation(name):
