@@ -107,6 +107,23 @@ fvattn_status_t fvattn_route(const void* q_r, const void* k_r, int32_t B, int32_
                              void* workspace, size_t workspace_bytes, fvattn_stream_t stream);
 
 /*
+ * Slack-aware sparse augmentation of a routed mask (Sec. 3.3, Eq. 8-9: a budget of extra blocks
+ * is spent by following the importance order routing already produced, and the mask is updated
+ * in place; no pooling, scoring or sorting is repeated).  Every query block of head (b,h) keeps
+ * the first counts[b,h,i] + extra[b,h] blocks of its importance order (score descending, ties to
+ * the lower index; clamped to nb) instead of the first counts[b,h,i]; mask_bits, counts, idx and
+ * head_load are rewritten accordingly, so the mask only grows.  extra[b,h] <= 0 leaves the head
+ * unchanged.  How a rank's slack becomes per-head budgets (Eq. 7-8) is the caller's business.
+ *   extra : i32 [B,H] on the device, blocks per query block.
+ *   workspace : the one the preceding fvattn_route used for this shape; its score matrix must
+ *               still be there (fvattn_sparse_attn and fvattn_tile_order leave it intact, another
+ *               fvattn_route overwrites it).
+ */
+fvattn_status_t fvattn_augment(int32_t B, int32_t H, int32_t d, const fvattn_grid_t* grid, const int32_t* extra,
+                               uint32_t* mask_bits, int32_t* counts, uint16_t* idx, float* head_load,
+                               void* workspace, size_t workspace_bytes, fvattn_stream_t stream);
+
+/*
  * Block-sparse attention over the retained (query block, key block) pairs (Sec. 2.1): for
  * each valid query row r of block i,
  *   O[r] = softmax_{r' in retained blocks, r' valid}(sm_scale * <Q[r],K[r']>) . V[r'],

@@ -298,6 +298,39 @@ void oracle_route(const uint16_t* q_r, const uint16_t* k_r, int32_t BH, int32_t 
 }
 
 /*
+ * Slack-aware sparse augmentation (Sec. 3.3; Eq. 8-9 give the budget, the step itself is "follow the
+ * importance order already produced by routing and add extra key blocks into the mask, in place").
+ * Reading: head bh gets extra[bh] more blocks for every one of its query blocks.  Row (bh, i) then keeps
+ * ranks 0 .. min(nb, counts + extra) - 1 of its importance order.
+ *   order  [BH, nb, nb]  importance order from oracle_route
+ *   counts [BH, nb]      in: current retained counts, out: augmented counts
+ *   extra  [BH]          blocks to add per query block (<= 0: unchanged)
+ * mask_bits and idx are rewritten for the augmented counts.
+ */
+void oracle_augment(const uint16_t* order, int32_t* counts, const int32_t* extra, int32_t BH, int32_t nb,
+                    uint32_t* mask_bits, uint16_t* idx) {
+    int32_t words = (nb + 31) / 32;
+    for (int32_t bh = 0; bh < BH; ++bh)
+        for (int32_t i = 0; i < nb; ++i) {
+            int64_t ri = (int64_t)bh * nb + i;
+            int32_t c = counts[ri] + (extra[bh] > 0 ? extra[bh] : 0);
+            if (c > nb) c = nb;
+            uint32_t* mb = mask_bits + ri * words;
+            for (int32_t w = 0; w < words; ++w) mb[w] = 0u;
+            for (int32_t m = 0; m < c; ++m) {
+                int32_t j = order[ri * nb + m];
+                mb[j >> 5] |= (1u << (j & 31));
+            }
+            uint16_t* ix = idx + ri * nb;
+            int32_t n_kept = 0;
+            for (int32_t j = 0; j < nb; ++j)
+                if (mb[j >> 5] & (1u << (j & 31))) ix[n_kept++] = (uint16_t)j;
+            for (int32_t m = n_kept; m < nb; ++m) ix[m] = 0xFFFFu;
+            counts[ri] = c;
+        }
+}
+
+/*
  * Block-sparse attention (Sec. 2.1: only selected pairs are evaluated), written
  * as the plain definition of masked softmax attention:
  *   for query row r of block i (head bh), over keys r' in the retained blocks

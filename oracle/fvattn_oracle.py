@@ -184,6 +184,22 @@ def route(q_r: np.ndarray, k_r: np.ndarray, g: Grid, p: float, k_floor: int, sm_
     return res
 
 
+def augment(res: RouteResult, extra: np.ndarray) -> RouteResult:
+    """Slack-aware augmentation (Sec. 3.3): head bh keeps extra[bh] more blocks per query block, taken in
+    the importance order (`res` must come from route(..., want_order=True)).  Returns a new RouteResult."""
+    assert res.order is not None
+    BH, nb = res.counts.shape
+    extra = np.ascontiguousarray(extra, dtype=np.int32)
+    assert extra.shape == (BH,)
+    counts = res.counts.copy()
+    mask_bits = np.empty_like(res.mask_bits)
+    idx = np.empty_like(res.idx)
+    lib().oracle_augment(_p(res.order), _p(counts), _p(extra), ctypes.c_int32(BH), ctypes.c_int32(nb),
+                         _p(mask_bits), _p(idx))
+    return RouteResult(mask_bits=mask_bits, counts=counts, idx=idx, head_load=counts.mean(-1).astype(np.float64),
+                       order=res.order, cum_at=res.cum_at, cum_before=res.cum_before, gap=res.gap)
+
+
 def sparse_attn(q_r: np.ndarray, k_r: np.ndarray, v_r: np.ndarray, idx: np.ndarray, counts: np.ndarray,
                 g: Grid, sm_scale: float, tiles: np.ndarray | None = None) -> np.ndarray:
     """Masked softmax attention over the retained blocks.

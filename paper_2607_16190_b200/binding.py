@@ -23,7 +23,8 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, E
 EXPORTS = (
     "fvattn_num_blocks", "fvattn_block_tokens", "fvattn_padded_tokens", "fvattn_workspace_bytes",
     "fvattn_workspace_init", "fvattn_reorder", "fvattn_inverse_reorder", "fvattn_route",
-    "fvattn_sparse_attn", "fvattn_sparse_attn_simt", "fvattn_sparse_attn_noalloc", "fvattn_tile_order", "fvattn_device_status",
+    "fvattn_augment", "fvattn_sparse_attn", "fvattn_sparse_attn_simt", "fvattn_sparse_attn_noalloc", "fvattn_tile_order",
+    "fvattn_device_status",
     "fvattn_status_string",
 )
 
@@ -204,6 +205,18 @@ def route(q_r: torch.Tensor, k_r: torch.Tensor, grid: Grid, p: float, k_floor: i
                               _ptr(out.counts), _ptr(out.idx), _ptr(out.head_load), _ptr(workspace),
                               ctypes.c_size_t(workspace.numel()), _stream()), "fvattn_route")
     return out
+
+
+def augment(routing: Routing, extra: torch.Tensor, grid: Grid, d: int, workspace: torch.Tensor) -> Routing:
+    """Slack-aware augmentation in place: head (b, h) keeps extra[b, h] more blocks per query block,
+    taken in the importance order of the preceding `route` call on this workspace."""
+    _need_cuda(extra, workspace, routing.counts)
+    B, H, nb = routing.counts.shape
+    assert extra.dtype == torch.int32 and extra.shape == (B, H) and extra.is_contiguous()
+    _check(lib().fvattn_augment(B, H, d, ctypes.byref(grid.c()), _ptr(extra), _ptr(routing.mask_bits),
+                                _ptr(routing.counts), _ptr(routing.idx), _ptr(routing.head_load), _ptr(workspace),
+                                ctypes.c_size_t(workspace.numel()), _stream()), "fvattn_augment")
+    return routing
 
 
 def _attn(fn_name: str, q_r, k_r, v_r, idx, counts, grid, sm_scale, workspace, out):

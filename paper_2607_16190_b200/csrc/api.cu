@@ -96,6 +96,22 @@ fvattn_status_t fvattn_route(const void* q_r, const void* k_r, int32_t B, int32_
                         workspace, (cudaStream_t)stream);
 }
 
+fvattn_status_t fvattn_augment(int32_t B, int32_t H, int32_t d, const fvattn_grid_t* grid, const int32_t* extra,
+                               uint32_t* mask_bits, int32_t* counts, uint16_t* idx, float* head_load, void* workspace,
+                               size_t workspace_bytes, fvattn_stream_t stream) {
+    if (!extra || !mask_bits || !counts || !idx || !workspace || !grid_ok(grid)) return FVATTN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0) return FVATTN_ERR_INVALID_ARG;
+    GridDims m = make_dims(*grid);
+    if (!shape_ok(d, m)) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if ((int64_t)B * H > 65535) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(workspace, 256) || !aligned(mask_bits, 4) || !aligned(counts, 4) || !aligned(idx, 2) ||
+        !aligned(extra, 4) || (head_load && !aligned(head_load, 4)))
+        return FVATTN_ERR_INVALID_ARG;
+    if (workspace_bytes < route_ws((int64_t)B * H, m.nb, d).total) return FVATTN_ERR_WORKSPACE_TOO_SMALL;
+    return launch_augment((int64_t)B * H, d, m, extra, mask_bits, counts, idx, head_load, workspace,
+                          (cudaStream_t)stream);
+}
+
 fvattn_status_t fvattn_tile_order(const int32_t* counts, int32_t B, int32_t H, const fvattn_grid_t* grid,
                                   uint32_t* order, void* workspace, size_t workspace_bytes, fvattn_stream_t stream) {
     if (!counts || !order || !workspace || !grid_ok(grid) || B <= 0 || H <= 0) return FVATTN_ERR_INVALID_ARG;

@@ -139,6 +139,8 @@ fvattn_status_t launch_inverse_reorder(const void* src_r, const GridDims& m, voi
 fvattn_status_t launch_route(const void* q_r, const void* k_r, int64_t BH, int d, const GridDims& m, float p,
                              int k_floor, float sm_scale, uint32_t* mask_bits, int32_t* counts, uint16_t* idx,
                              float* head_load, void* workspace, cudaStream_t s);
+fvattn_status_t launch_augment(int64_t BH, int d, const GridDims& m, const int32_t* extra, uint32_t* mask_bits,
+                               int32_t* counts, uint16_t* idx, float* head_load, void* workspace, cudaStream_t s);
 fvattn_status_t launch_tile_order(const int32_t* counts, int64_t BH, int nb, uint32_t* order, void* workspace,
                                   cudaStream_t s);
 fvattn_status_t launch_attn_simt(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,

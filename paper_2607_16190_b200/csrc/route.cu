@@ -295,7 +295,8 @@ __device__ __forceinline__ float block_sum(float v, float* red) {
 // dynamic smem: keys u64[n2] | prob f32[n2] | sorted prob f32[n2] | bits u32[n2/32] | wpre u32[n2/32]
 __global__ void __launch_bounds__(kSelThreads)
 select_kernel(const float* __restrict__ scores, int nb, int n2, int score_stride, float p, int k_floor,
-              uint32_t* __restrict__ mask_bits, int32_t* __restrict__ counts, uint16_t* __restrict__ idx) {
+              uint32_t* __restrict__ mask_bits, int32_t* counts, uint16_t* __restrict__ idx,
+              const int32_t* __restrict__ extra) {
     extern __shared__ __align__(16) unsigned char smem_raw[];
     unsigned long long* keys = reinterpret_cast<unsigned long long*>(smem_raw);
     float* prob = reinterpret_cast<float*>(keys + n2);
@@ -384,7 +385,8 @@ select_kernel(const float* __restrict__ scores, int nb, int n2, int score_stride
         }
     }
     __syncthreads();
-    const int c = max(cut, min(k_floor, nb));
+    const int c = extra ? min(nb, max(1, counts[row] + max(extra[row / nb], 0))) : max(cut, min(k_floor, nb));
+    __syncthreads();   // every thread has read counts[row] before thread 0 overwrites it
 
     // materialise: bit mask, ascending index list, count
     for (int m_ = tid; m_ < c; m_ += kSelThreads) {
@@ -444,7 +446,8 @@ __device__ __forceinline__ int warp_sum(int v) {
 template <int E>
 __global__ void __launch_bounds__(kSelWarpsPerCta * 32)
 select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int score_stride, float p, int k_floor,
-                   uint32_t* __restrict__ mask_bits, int32_t* __restrict__ counts, uint16_t* __restrict__ idx) {
+                   uint32_t* __restrict__ mask_bits, int32_t* counts, uint16_t* __restrict__ idx,
+                   const int32_t* __restrict__ extra /* NULL, or per head: blocks to add to each row's count */) {
     __shared__ uint32_t hist[kSelWarpsPerCta * 512];
     const int lane = threadIdx.x & 31;
     const int64_t row = (int64_t)blockIdx.x * kSelWarpsPerCta + (threadIdx.x >> 5);
@@ -485,7 +488,13 @@ select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int
 #pragma unroll
     for (int e = 0; e < E; ++e) mass_fx[e] = __float2uint_rn(sc[e] * to_fx);
 
-    const int need_cnt = max(1, min(k_floor, nb));
+    // routing: mass >= p and at least the floor; augmentation (Sec. 3.3): exactly the row's current count
+    // plus the head's extra blocks, taken further down the same importance order
+    int need_cnt = max(1, min(k_floor, nb));
+    if (extra) {
+        need_cnt = min(nb, max(1, counts[row] + max(extra[row / nb], 0)));
+        p = 0.f;
+    }
     const uint32_t p_fx = p > 0.f ? __float2uint_ru(p * 2147483648.0f) : 0u;
     uint32_t thr = 0xffffffffu;          // p >= 1 keeps everything
     int r_ties = 1 << 30;                // how many blocks with key == thr are kept (index order)
@@ -627,10 +636,10 @@ select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int
 template <int E>
 static fvattn_status_t launch_select_warp(const float* scores, int nb, int64_t n_rows, int score_stride, float p,
                                           int k_floor, uint32_t* mask_bits, int32_t* counts, uint16_t* idx,
-                                          cudaStream_t s) {
+                                          const int32_t* extra, cudaStream_t s) {
     const unsigned ctas = (unsigned)((n_rows + kSelWarpsPerCta - 1) / kSelWarpsPerCta);
     select_warp_kernel<E><<<ctas, kSelWarpsPerCta * 32, 0, s>>>(scores, nb, n_rows, score_stride, p, k_floor,
-                                                                  mask_bits, counts, idx);
+                                                                  mask_bits, counts, idx, extra);
     return launch_status();
 }
 
@@ -709,6 +718,31 @@ static fvattn_status_t launch_stages(const void* q_r, const void* k_r, int64_t B
     return launch_status();
 }
 
+// Selection over the score matrix: routing (extra == NULL) or augmentation of an existing mask.
+static fvattn_status_t launch_selection(const float* scores, int64_t BH, const GridDims& m, int score_stride, float p,
+                                        int k_floor, uint32_t* mask_bits, int32_t* counts, uint16_t* idx,
+                                        const int32_t* extra, cudaStream_t s) {
+    const int64_t n_rows = BH * m.nb;
+    fvattn_status_t st;
+    if (m.nb <= 1024) {
+        const int e = (m.nb + 31) / 32;
+#define FVATTN_SEL_CASE(E_) \
+    if (e <= E_) st = launch_select_warp<E_>(scores, m.nb, n_rows, score_stride, p, k_floor, mask_bits, counts, idx, extra, s); else
+        FVATTN_SEL_CASE(1) FVATTN_SEL_CASE(4) FVATTN_SEL_CASE(8) FVATTN_SEL_CASE(12) FVATTN_SEL_CASE(16)
+        FVATTN_SEL_CASE(20) FVATTN_SEL_CASE(24) FVATTN_SEL_CASE(28)
+        st = launch_select_warp<32>(scores, m.nb, n_rows, score_stride, p, k_floor, mask_bits, counts, idx, extra, s);
+#undef FVATTN_SEL_CASE
+        return st;
+    }
+    int n2 = 2048;
+    while (n2 < m.nb) n2 <<= 1;
+    const size_t smem = (size_t)n2 * (8 + 4 + 4) + 2 * sizeof(uint32_t) * (size_t)(n2 / 32);
+    FVATTN_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    select_kernel<<<(unsigned)n_rows, kSelThreads, smem, s>>>(scores, m.nb, n2, score_stride, p, k_floor, mask_bits,
+                                                             counts, idx, extra);
+    return launch_status();
+}
+
 fvattn_status_t launch_route(const void* q_r, const void* k_r, int64_t BH, int d, const GridDims& m, float p,
                              int k_floor, float sm_scale, uint32_t* mask_bits, int32_t* counts, uint16_t* idx,
                              float* head_load, void* workspace, cudaStream_t s) {
@@ -727,26 +761,26 @@ fvattn_status_t launch_route(const void* q_r, const void* k_r, int64_t BH, int d
                                                       sms, workspace, s);
     if (st != FVATTN_OK) return st;
 
-    const int64_t n_rows = BH * m.nb;
-    if (m.nb <= 1024) {
-        const int e = (m.nb + 31) / 32;
-#define FVATTN_SEL_CASE(E_) \
-    if (e <= E_) st = launch_select_warp<E_>(scores, m.nb, n_rows, w.score_stride, p, k_floor, mask_bits, counts, idx, s); else
-        FVATTN_SEL_CASE(1) FVATTN_SEL_CASE(4) FVATTN_SEL_CASE(8) FVATTN_SEL_CASE(12) FVATTN_SEL_CASE(16)
-        FVATTN_SEL_CASE(20) FVATTN_SEL_CASE(24) FVATTN_SEL_CASE(28)
-        st = launch_select_warp<32>(scores, m.nb, n_rows, w.score_stride, p, k_floor, mask_bits, counts, idx, s);
-#undef FVATTN_SEL_CASE
-        if (st != FVATTN_OK) return st;
-    } else {
-        int n2 = 2048;
-        while (n2 < m.nb) n2 <<= 1;
-        const size_t smem = (size_t)n2 * (8 + 4 + 4) + 2 * sizeof(uint32_t) * (size_t)(n2 / 32);
-        FVATTN_CUDA_OK(cudaFuncSetAttribute(select_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        select_kernel<<<(unsigned)n_rows, kSelThreads, smem, s>>>(scores, m.nb, n2, w.score_stride, p, k_floor,
-                                                                 mask_bits, counts, idx);
+    st = launch_selection(scores, BH, m, w.score_stride, p, k_floor, mask_bits, counts, idx, nullptr, s);
+    if (st != FVATTN_OK) return st;
+
+    if (head_load) {
+        head_load_kernel<<<(unsigned)BH, 256, 0, s>>>(counts, m.nb, head_load);
         if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
     }
+    return FVATTN_OK;
+}
 
+// Slack-aware augmentation (Sec. 3.3): every query block of head bh keeps its first
+// counts + extra[bh] blocks of the importance order instead of its first counts.  The order is
+// the one the score matrix of the preceding fvattn_route defines (still in the workspace), so no
+// pooling, scoring or sorting is repeated.
+fvattn_status_t launch_augment(int64_t BH, int d, const GridDims& m, const int32_t* extra, uint32_t* mask_bits,
+                               int32_t* counts, uint16_t* idx, float* head_load, void* workspace, cudaStream_t s) {
+    RouteWs w = route_ws(BH, m.nb, d);
+    const float* scores = reinterpret_cast<const float*>(static_cast<char*>(workspace) + w.scores);
+    fvattn_status_t st = launch_selection(scores, BH, m, w.score_stride, 0.f, 0, mask_bits, counts, idx, extra, s);
+    if (st != FVATTN_OK) return st;
     if (head_load) {
         head_load_kernel<<<(unsigned)BH, 256, 0, s>>>(counts, m.nb, head_load);
         if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;

@@ -258,6 +258,32 @@ def test_hand_worked_rows():
             assert res.idx[0, i, :len(kept)].tolist() == kept, (case, i)
 
 
+# ---------------------------------------------------------------- augmentation (Sec. 3.3)
+def test_augmentation_appends_the_next_ranks_and_only_grows_the_mask():
+    cfg, g, q_r, k_r, _ = _routing_inputs("small")
+    nb = O.num_blocks(g)
+    res = O.route(q_r, k_r, g, 0.5, 1, cfg.sm_scale, want_order=True)
+    extra = np.array([0, 1, 2, 3, nb, -4, 5, 0, 1, 7, 2, 100], dtype=np.int32)
+    aug = O.augment(res, extra)
+    M0, M1 = res.mask_bool(), aug.mask_bool()
+    assert (M1 | M0 == M1).all()                                   # the mask only grows
+    want_counts = np.minimum(nb, res.counts + np.maximum(extra, 0)[:, None])
+    np.testing.assert_array_equal(aug.counts, want_counts)
+    assert (M1.sum(-1) == want_counts).all()
+    # independent statement: the kept set is the top (count + extra) of a stable numpy argsort of the scores
+    s, _ = _independent_probs(q_r, k_r, g, cfg.sm_scale)
+    rank = np.argsort(np.argsort(-s, axis=-1, kind="stable"), axis=-1, kind="stable")
+    np.testing.assert_array_equal(M1, rank < want_counts[..., None])
+    for h in range(M1.shape[0]):
+        for i in range(nb):
+            c = want_counts[h, i]
+            assert aug.idx[h, i, :c].tolist() == np.nonzero(M1[h, i])[0].tolist()
+            assert (aug.idx[h, i, c:] == 0xFFFF).all()
+    np.testing.assert_allclose(aug.head_load, want_counts.mean(-1))   # Eq. 1 on the augmented mask
+    # heads with no budget are untouched
+    np.testing.assert_array_equal(aug.mask_bits[[0, 5, 7]], res.mask_bits[[0, 5, 7]])
+
+
 # ---------------------------------------------------------------- attention (Sec. 2.1)
 def _dense_attention_tokens(q, k, v, sm_scale):
     """Brute-force softmax attention on the ORIGINAL token order: q,k,v [N, H, d] f64."""
