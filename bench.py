@@ -379,7 +379,7 @@ def run_sweep(args):
     import torch
 
     from paper_2607_16190_b200 import binding as fv
-    from paper_2607_16190_b200 import synth
+    from paper_2607_16190_b200 import planner, synth
 
     torch.cuda.set_device(0)
     base = synth.CONFIGS["wan720p"]
@@ -389,6 +389,7 @@ def run_sweep(args):
     full = None
     acc = {p: {"density": [], "route_ms": [], "attn_ms": []} for p in synth.SWEEP_P}
     dense_own, dense_sdpa = [], []
+    virt = {k_: [] for k_ in ("rho_before", "rho_after_rlb", "rho_after_sasa", "augment_ms", "density_after_sasa")}
     for li in range(args.sweep_layers):
         cfg = synth.sweep_layer(li)
         q, k, v, _ = synth.make_qkv(cfg, "cuda:0")
@@ -405,6 +406,19 @@ def run_sweep(args):
             acc[p]["route_ms"].append(time_steps(route, 1, torch))
             acc[p]["attn_ms"].append(time_steps(attn, 1, torch))
             acc[p]["density"].append(int(layer.routing.counts.sum().item()) / (cfg.H * nb * nb))
+            if p == 0.9:
+                # virtual 8-rank Ulysses layout (context for the paper's 1.34 -> 1.08): imbalance before and
+                # after the constrained head migration, then slack budgets spent by fvattn_augment
+                loads = layer.routing.head_load[0].double().cpu().numpy()
+                plan = planner.plan_migration(loads, 8)
+                extra, _, aug_loads = planner.slack_budgets(plan.loads_after, planner.heads_after(plan, cfg.H), cfg.H)
+                ex = torch.from_numpy(extra).to("cuda:0")[None].contiguous()
+                t_aug = time_steps(lambda: fv.augment(layer.routing, ex, g, cfg.d, layer.workspace), 1, torch)
+                virt["rho_before"].append(plan.rho_before)
+                virt["rho_after_rlb"].append(plan.rho_after)
+                virt["rho_after_sasa"].append(planner.imbalance(aug_loads))
+                virt["augment_ms"].append(t_aug)
+                virt["density_after_sasa"].append(int(layer.routing.counts.sum().item()) / (cfg.H * nb * nb))
         if li < args.sweep_dense_layers:                      # dense baselines on the same inputs
             full = fv.route(layer.q_r, layer.k_r, g, 1.0, cfg.k_floor, layer.sm_scale, layer.workspace, full)
             own = lambda: fv.sparse_attn(layer.q_r, layer.k_r, layer.v_r, full.idx, full.counts, g, layer.sm_scale,
@@ -428,7 +442,8 @@ def run_sweep(args):
                      "speedup_vs_dense_own_kernel": mean(dense_own) / mean(a["attn_ms"]),
                      "speedup_vs_dense_sdpa": mean(dense_sdpa) / mean(a["attn_ms"])})
     print(json.dumps({"sweep": "wan720p x %d layers" % args.sweep_layers, "device_status": fv.status_string(status),
-                      "dense_own_kernel_ms": mean(dense_own), "dense_sdpa_ms": mean(dense_sdpa), "rows": rows}), flush=True)
+                      "dense_own_kernel_ms": mean(dense_own), "dense_sdpa_ms": mean(dense_sdpa), "rows": rows,
+                      "virtual_8_ranks_p0.9": {k_: mean(v_) for k_, v_ in virt.items()}}), flush=True)
 
 
 def main():

@@ -1,0 +1,146 @@
+"""Host-side workload planner over VIRTUAL ranks: the paper's load metrics, the constrained
+head-migration search and the slack budgets, evaluated on the per-head loads `fvattn_route`
+returns.  Nothing here touches a GPU or moves data: on one GPU the ranks are a simulation that
+(a) reports the imbalance a Ulysses layout would see and (b) turns slack into the per-head
+budgets `fvattn_augment` spends.  Deterministic: the same loads give the same plan everywhere.
+
+Passages: Eq. 1-2 (L_r, rho), Eq. 5-6 (one-send-one-receive migration, lexicographic
+objective (max load, variance)), Eq. 7-9 (slack, budget, augmented load), the piecewise enable
+policy of Sec. 3.3.  Readings where the paper is silent: heads are laid out in Ulysses order
+(rank r owns heads [r*H/R, (r+1)*H/R)); the candidate space is the set of pair topologies
+(involutions of the ranks: a matched pair swaps one head each way, unmatched ranks keep their
+heads); per pair the swap minimising (pair max, pair sum of squares) is taken; a rank's budget is
+split evenly over its heads and rounded down to whole blocks per query block.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+
+def rank_loads(head_load: np.ndarray, ranks: int) -> np.ndarray:
+    """L_r = sum of L_h over the rank's heads (Eq. 1), heads in Ulysses order."""
+    L = np.asarray(head_load, dtype=np.float64)
+    assert L.ndim == 1 and L.size % ranks == 0
+    return L.reshape(ranks, -1).sum(1)
+
+
+def imbalance(loads: np.ndarray) -> float:
+    """rho = max_r L_r / mean_r L_r (Eq. 2)."""
+    loads = np.asarray(loads, dtype=np.float64)
+    return float(loads.max() / loads.mean())
+
+
+def _involutions(n: int):
+    """All pairings of range(n) with any number of unmatched elements, in a fixed order."""
+    def rec(free):
+        if not free:
+            yield []
+            return
+        a, rest = free[0], free[1:]
+        yield from rec(rest)                                   # a stays unmatched
+        for k, b in enumerate(rest):
+            for tail in rec(rest[:k] + rest[k + 1:]):
+                yield [(a, b)] + tail
+    yield from rec(list(range(n)))
+
+
+@dataclass
+class MigrationPlan:
+    sigma: list                      # sigma[r] = rank that r sends to (r itself: no migration)
+    sent_head: list                  # global head index r sends, or -1
+    loads_before: np.ndarray
+    loads_after: np.ndarray
+    rho_before: float = field(init=False)
+    rho_after: float = field(init=False)
+
+    def __post_init__(self):
+        self.rho_before, self.rho_after = imbalance(self.loads_before), imbalance(self.loads_after)
+
+
+def _best_swap(Li, Lj, heads_i, heads_j):
+    """Swap one head each way between two ranks: minimise (max, sum of squares), first best wins."""
+    best = (max(Li, Lj), Li * Li + Lj * Lj, -1, -1)
+    for a, la in enumerate(heads_i):
+        for b, lb in enumerate(heads_j):
+            ni, nj = Li - la + lb, Lj - lb + la                # Eq. 5
+            cand = (max(ni, nj), ni * ni + nj * nj, a, b)
+            if cand[:2] < best[:2]:
+                best = cand
+    return best
+
+
+def plan_migration(head_load: np.ndarray, ranks: int) -> MigrationPlan:
+    """Eq. 6 over pair topologies: every rank sends at most one head and receives at most one.
+    Exhaustive over involutions for ranks <= 8 (764 of them at 8), greedy heaviest-with-lightest
+    pairing above that."""
+    L = np.asarray(head_load, dtype=np.float64)
+    per = L.size // ranks
+    heads = L.reshape(ranks, per)
+    loads = heads.sum(1)
+    swap = {}
+    for i in range(ranks):
+        for j in range(i + 1, ranks):
+            swap[(i, j)] = _best_swap(loads[i], loads[j], heads[i], heads[j])
+    if ranks <= 8:
+        candidates = _involutions(ranks)
+    else:
+        order = np.argsort(-loads, kind="stable")
+        candidates = [[(min(order[k], order[-1 - k]), max(order[k], order[-1 - k])) for k in range(ranks // 2)], []]
+    best_key, best_pairs = None, []
+    for pairs in candidates:
+        new = loads.copy()
+        for (i, j) in pairs:
+            mx, _, a, b = swap[(i, j)]
+            if a >= 0:
+                new[i] += heads[j, b] - heads[i, a]
+                new[j] += heads[i, a] - heads[j, b]
+        key = (float(new.max()), float(new.var()))
+        if best_key is None or key < best_key:
+            best_key, best_pairs = key, list(pairs)
+    sigma, sent = list(range(ranks)), [-1] * ranks
+    after = loads.copy()
+    for (i, j) in best_pairs:
+        _, _, a, b = swap[(i, j)]
+        if a >= 0:
+            sigma[i], sigma[j] = j, i
+            sent[i], sent[j] = i * per + a, j * per + b
+            after[i] += heads[j, b] - heads[i, a]
+            after[j] += heads[i, a] - heads[j, b]
+    return MigrationPlan(sigma, sent, loads, after)
+
+
+def heads_after(plan: MigrationPlan, n_heads: int) -> list:
+    """Heads resident on each rank once the plan's migrations are done."""
+    ranks = len(plan.sigma)
+    per = n_heads // ranks
+    res = [list(range(r * per, (r + 1) * per)) for r in range(ranks)]
+    for r, h in enumerate(plan.sent_head):
+        if h >= 0:
+            res[r].remove(h)
+            res[plan.sigma[r]].append(h)
+    return res
+
+
+def slack_budgets(loads: np.ndarray, rank_heads: list, n_heads: int, n1: float = 0.8, n2: float = 0.07):
+    """Eq. 7-9.  `rank_heads[r]` lists the heads on rank r.  Returns (extra blocks per query block for
+    each head [n_heads] int32, B_r, augmented loads).  A rank is augmented only if its slack exceeds
+    n2 * L_max; its budget is split evenly over its heads and rounded down to whole blocks."""
+    loads = np.asarray(loads, dtype=np.float64)
+    lmax = loads.max()
+    slack = lmax - loads                                       # Eq. 7
+    budget = np.where(slack > n2 * lmax, n1 * slack, 0.0)      # Eq. 8 with the trigger
+    extra = np.zeros(n_heads, dtype=np.int32)
+    aug = loads.copy()
+    for r, hs in enumerate(rank_heads):
+        if hs:
+            e = int(np.floor(budget[r] / len(hs)))
+            extra[hs] = e
+            aug[r] += e * len(hs)                              # Eq. 9 with the rounded budget
+    return extra, budget, aug
+
+
+def enable_policy(rho: float, k1: float = 1.05, k2: float = 1.10) -> str:
+    """Piecewise policy of Sec. 3.3: 'none' below k1, 'sasa' in [k1, k2), 'rlb+sasa' from k2."""
+    return "none" if rho < k1 else ("sasa" if rho < k2 else "rlb+sasa")

@@ -1,0 +1,94 @@
+"""Host-side planner over virtual ranks (Eq. 1-2, 5-9): closed forms and brute force."""
+import itertools
+
+import numpy as np
+
+from paper_2607_16190_b200 import planner as P
+
+
+def test_rank_loads_and_rho_closed_forms():
+    L = np.array([1, 2, 3, 4, 5, 6, 7, 8], dtype=float)
+    np.testing.assert_array_equal(P.rank_loads(L, 4), [3, 7, 11, 15])      # Ulysses order, Eq. 1
+    assert P.imbalance([3, 7, 11, 15]) == 15 / 9                            # Eq. 2
+    assert P.imbalance([5, 5, 5]) == 1.0
+
+
+def _brute_force_min_max(heads):
+    """Every involution of the ranks and every choice of swapped heads (or no swap) per pair."""
+    R, per = heads.shape
+    loads = heads.sum(1)
+    best = loads.max()
+
+    def rec(free, new):
+        nonlocal best
+        if not free:
+            best = min(best, new.max())
+            return
+        a, rest = free[0], free[1:]
+        rec(rest, new)
+        for k, b in enumerate(rest):
+            others = rest[:k] + rest[k + 1:]
+            for ha, hb in itertools.product(range(per), range(per)):
+                n2 = new.copy()
+                n2[a] += heads[b, hb] - heads[a, ha]
+                n2[b] += heads[a, ha] - heads[b, hb]
+                rec(others, n2)
+    rec(list(range(R)), loads.astype(float).copy())
+    return best
+
+
+def test_plan_reaches_the_brute_force_critical_path_and_respects_the_constraint():
+    rng = np.random.default_rng(0)
+    for trial in range(6):
+        R, per = 4, 3
+        heads = np.exp(rng.normal(0, 1.0, size=(R, per))) * 20
+        plan = P.plan_migration(heads.reshape(-1), R)
+        assert abs(plan.loads_after.max() - _brute_force_min_max(heads)) < 1e-9
+        # one send, one receive, at most one head per rank; sigma is an involution here
+        assert sorted(plan.sigma) == list(range(R))
+        for r in range(R):
+            assert plan.sigma[plan.sigma[r]] == r
+            assert (plan.sent_head[r] >= 0) == (plan.sigma[r] != r)
+            if plan.sent_head[r] >= 0:
+                assert plan.sent_head[r] // per == r
+        # Eq. 5 recomputed from the plan
+        want = heads.sum(1).copy()
+        flat = heads.reshape(-1)
+        for r in range(R):
+            if plan.sent_head[r] >= 0:
+                want[r] -= flat[plan.sent_head[r]]
+                want[plan.sigma[r]] += flat[plan.sent_head[r]]
+        np.testing.assert_allclose(plan.loads_after, want)
+        assert plan.rho_after <= plan.rho_before + 1e-12
+        np.testing.assert_allclose(plan.loads_after.sum(), plan.loads_before.sum())
+        after = P.heads_after(plan, R * per)
+        assert sorted(h for hs in after for h in hs) == list(range(R * per))
+        np.testing.assert_allclose([flat[hs].sum() for hs in after], plan.loads_after)
+
+
+def test_balanced_loads_need_no_migration_and_eight_ranks_run():
+    plan = P.plan_migration(np.full(40, 3.0), 8)
+    assert plan.sigma == list(range(8)) and plan.rho_after == 1.0
+    rng = np.random.default_rng(1)
+    L = np.exp(rng.normal(0.5, 0.8, size=40)).clip(0.3, 8) * 50
+    plan = P.plan_migration(L, 8)
+    assert plan.rho_after <= plan.rho_before
+    plan16 = P.plan_migration(np.tile(L, 2), 16)              # greedy path above 8 ranks
+    assert plan16.rho_after <= plan16.rho_before + 1e-12
+
+
+def test_slack_budgets_eq_7_to_9():
+    loads = np.array([100.0, 90.0, 60.0, 96.0])
+    rank_heads = [[0, 1], [2, 3], [4, 5], [6, 7]]
+    extra, budget, aug = P.slack_budgets(loads, rank_heads, 8, n1=0.8, n2=0.07)
+    # slack = 0, 10, 40, 4; trigger 0.07 * 100 = 7 -> ranks 1 and 2; B = 8, 32
+    np.testing.assert_allclose(budget, [0, 8, 32, 0])
+    assert extra.tolist() == [0, 0, 4, 4, 16, 16, 0, 0]
+    np.testing.assert_allclose(aug, [100, 98, 92, 96])
+    assert aug.max() <= loads.max()                            # no new straggler
+
+
+def test_enable_policy_thresholds():
+    assert P.enable_policy(1.04) == "none"
+    assert P.enable_policy(1.05) == "sasa" and P.enable_policy(1.0999) == "sasa"
+    assert P.enable_policy(1.10) == "rlb+sasa" and P.enable_policy(1.34) == "rlb+sasa"
