@@ -47,6 +47,7 @@ pool_kernel(const uint4* __restrict__ q_r, const uint4* __restrict__ k_r, __nv_b
     const uint32_t block_bytes = (uint32_t)m.bs * D * 2;
     float* partial = reinterpret_cast<float*>(pool_smem + (size_t)kPoolStages * block_bytes);   // [2][RG][D]
     unsigned short* vcount = reinterpret_cast<unsigned short*>(partial + 2 * RG * D);           // [nb] valid rows
+    unsigned short* vrows = vcount + m.nb;   // [nb] rows to fetch: up to and including the last valid row
     __shared__ unsigned long long full[kPoolStages];
     __shared__ int abort_flag;
 
@@ -57,7 +58,12 @@ pool_kernel(const uint4* __restrict__ q_r, const uint4* __restrict__ k_r, __nv_b
     const int64_t my_items = first < n_items ? (n_items - first + stride - 1) / stride : 0;
     const int64_t part_stride = per_tensor * D;                     // elements between the hi / mid / lo planes
 
-    for (int b = tid; b < m.nb; b += kPoolThreads) vcount[b] = (unsigned short)block_valid_tokens(m, b);
+    for (int b = tid; b < m.nb; b += kPoolThreads) {
+        vcount[b] = (unsigned short)block_valid_tokens(m, b);
+        const int bx = b % m.nX, by = (b / m.nX) % m.nY, bt = b / (m.nX * m.nY);
+        const int vt = min(m.tT, m.T - bt * m.tT), vy = min(m.tY, m.Y - by * m.tY), vx = min(m.tX, m.X - bx * m.tX);
+        vrows[b] = (unsigned short)(((vt - 1) * m.tY + (vy - 1)) * m.tX + vx);   // trailing padding rows are not read
+    }
     if (tid == 0) {
         for (int s = 0; s < kPoolStages; ++s) mbar_init(smem_u32(&full[s]), 1);
         abort_flag = 0;
@@ -71,8 +77,9 @@ pool_kernel(const uint4* __restrict__ q_r, const uint4* __restrict__ k_r, __nv_b
         const uint4* src = (item >= per_tensor ? k_r : q_r) + rest * (int64_t)m.bs * VPR;
         const int s = (int)(k % kPoolStages);
         const uint32_t bar = smem_u32(&full[s]);
-        mbar_expect_tx(bar, block_bytes);
-        bulk_load_1d(smem_u32(pool_smem + (size_t)s * block_bytes), src, block_bytes, bar);
+        const uint32_t bytes = (uint32_t)vrows[(uint32_t)rest % (uint32_t)m.nb] * (D * 2);
+        mbar_expect_tx(bar, bytes);
+        bulk_load_1d(smem_u32(pool_smem + (size_t)s * block_bytes), src, bytes, bar);
     };
     if (tid == 0)
         for (int64_t k = 0; k < kPoolStages - 1 && k < my_items; ++k) issue(k);
@@ -432,6 +439,12 @@ select_kernel(const float* __restrict__ scores, int nb, int n2, int score_stride
 // prefix pop-counts give the ascending compact index list.
 constexpr int kSelWarpsPerCta = 8;
 
+// 2^x on the special-function unit (relative error about 2^-22: below the fp32 rounding of the masses)
+__device__ __forceinline__ float exp2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -480,7 +493,7 @@ select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int
     for (int e = 0; e < E; ++e) {
         const int j = lane + 32 * e;
         key[e] = (j < nb) ? min(__float2uint_rn((mx - sc[e]) * key_scale), 268435455u) : 0xffffffffu;
-        sc[e] = (j < nb) ? expf(sc[e] - mx) : 0.f;
+        sc[e] = (j < nb) ? exp2_approx((sc[e] - mx) * 1.4426950408889634f) : 0.f;
         z += sc[e];
     }
     z = warp_sum(z);
@@ -614,21 +627,36 @@ select_warp_kernel(const float* __restrict__ scores, int nb, int64_t n_rows, int
     // materialise
     uint32_t* mrow = mask_bits + row * ((nb + 31) / 32);
     uint16_t* irow = idx + row * nb;
-    int base = 0, ties_seen = 0;
+    int base = 0;
+    if (r_ties == (1 << 30)) {               // no tie group is split: the kept set is {key <= thr}
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-        const int j = lane + 32 * e;
-        const bool eq = key[e] == thr && j < nb;
-        const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
-        const int tie_rank = ties_seen + __popc(eq_ballot & ((1u << lane) - 1u));
-        ties_seen += __popc(eq_ballot);
-        const bool keep = j < nb && (key[e] < thr || (eq && tie_rank < r_ties));
-        const uint32_t word = __ballot_sync(0xffffffffu, keep);
-        if (32 * e < nb) {
-            if (lane == 0) mrow[e] = word;
-            if (keep) irow[base + __popc(word & ((1u << lane) - 1u))] = (uint16_t)j;
+        for (int e = 0; e < E; ++e) {
+            const int j = lane + 32 * e;
+            const bool keep = j < nb && key[e] <= thr;
+            const uint32_t word = __ballot_sync(0xffffffffu, keep);
+            if (32 * e < nb) {
+                if (lane == 0) mrow[e] = word;
+                if (keep) irow[base + __popc(word & ((1u << lane) - 1u))] = (uint16_t)j;
+            }
+            base += __popc(word);
         }
-        base += __popc(word);
+    } else {
+        int ties_seen = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const int j = lane + 32 * e;
+            const bool eq = key[e] == thr && j < nb;
+            const uint32_t eq_ballot = __ballot_sync(0xffffffffu, eq);
+            const int tie_rank = ties_seen + __popc(eq_ballot & ((1u << lane) - 1u));
+            ties_seen += __popc(eq_ballot);
+            const bool keep = j < nb && (key[e] < thr || (eq && tie_rank < r_ties));
+            const uint32_t word = __ballot_sync(0xffffffffu, keep);
+            if (32 * e < nb) {
+                if (lane == 0) mrow[e] = word;
+                if (keep) irow[base + __popc(word & ((1u << lane) - 1u))] = (uint16_t)j;
+            }
+            base += __popc(word);
+        }
     }
     if (lane == 0) counts[row] = base;
 }
@@ -700,7 +728,7 @@ static fvattn_status_t launch_stages(const void* q_r, const void* k_r, int64_t B
                                      int sms, void* workspace, cudaStream_t s) {
     {
         const size_t block_bytes = (size_t)m.bs * D * 2;
-        const size_t smem = kPoolStages * block_bytes + 2 * sizeof(float) * kPoolThreads * 8 + 2 * (size_t)m.nb;
+        const size_t smem = kPoolStages * block_bytes + 2 * sizeof(float) * kPoolThreads * 8 + 4 * (size_t)m.nb;
         const int64_t items = 2 * BH * m.nb;
         const unsigned grid = (unsigned)(items < sms * kPoolCtasPerSm ? items : sms * kPoolCtasPerSm);
         FVATTN_CUDA_OK(cudaFuncSetAttribute(pool_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
