@@ -86,6 +86,31 @@ fvattn_status_t fvattn_inverse_reorder(const void* src_r, const fvattn_grid_t* g
                                        fvattn_tok_layout_t lay, fvattn_stream_t stream);
 
 /*
+ * Table-driven block organisation, and the Hilbert-curve table (Sec. 3.1: "reorders blocks along
+ * a Hilbert curve so that spatially adjacent tokens tend to fall into nearby blocks").
+ *
+ * fvattn_hilbert_row_tokens (host arithmetic, host pointers): row_token[r] = index of the token
+ * (raster order over T,Y,X) that sits at position r of the 3-D Hilbert curve through the grid
+ * (the curve of the enclosing power-of-two cube, restricted to the grid's cells); rows past the
+ * last token are -1.  n_rows must be ceil(T*Y*X / block_tokens) * block_tokens.  Blocks are
+ * block_tokens consecutive curve positions; only the last block has padding.
+ *
+ * fvattn_reorder_by_table / fvattn_inverse_reorder_by_table: as fvattn_reorder /
+ * fvattn_inverse_reorder with the row -> token map given as a DEVICE table row_token
+ * [ceil(n_tokens / block_tokens) * block_tokens] (entries outside [0, n_tokens) are padding; every
+ * token must appear once).  Downstream, fvattn_route / fvattn_sparse_attn / fvattn_augment take
+ * this layout as the 1-D grid {T=1, Y=1, X=n_tokens, tT=1, tY=1, tX=block_tokens}.
+ */
+fvattn_status_t fvattn_hilbert_row_tokens(int32_t T, int32_t Y, int32_t X, int32_t block_tokens,
+                                          int32_t* row_token /* host */, int64_t n_rows);
+fvattn_status_t fvattn_reorder_by_table(const void* src, fvattn_tok_layout_t lay, const int32_t* row_token,
+                                        int64_t n_tokens, int32_t block_tokens, void* dst_r,
+                                        fvattn_stream_t stream);
+fvattn_status_t fvattn_inverse_reorder_by_table(const void* src_r, const int32_t* row_token, int64_t n_tokens,
+                                                int32_t block_tokens, void* dst, fvattn_tok_layout_t lay,
+                                                fvattn_stream_t stream);
+
+/*
  * Top-p block routing with a Top-k floor (Sec. 2.1; Sec. 3.1 pooled similarities; Eq. 1).
  * For every head bh and query block i:
  *   qbar, kbar = mean of the block's valid (non-padding) rows          (fp32)

@@ -409,3 +409,50 @@ void oracle_sparse_attn(const uint16_t* q_r, const uint16_t* k_r, const uint16_t
     }
     free(valid);
 }
+
+/*
+ * Hilbert-curve block organisation (Sec. 3.1: blocks follow a Hilbert curve so that spatially
+ * adjacent tokens fall into nearby blocks).  Reading: the 3-D Hilbert curve of the smallest
+ * power-of-two cube that holds the (T, Y, X) grid is walked from its start, index by index, and
+ * the cells that belong to the grid are taken in the order met; row r of the reordered sequence
+ * holds the r-th such token (raster index over T, Y, X), rows past the last token hold -1.
+ * The walk maps each curve index to its cell (de-interleave, Gray decode, redo the rotations from
+ * the low bit plane up); nothing is sorted.
+ */
+static void hilbert_cell(uint64_t h, int bits, uint32_t c[3]) {
+    uint32_t x[3] = {0u, 0u, 0u};
+    for (int b = bits - 1; b >= 0; --b)
+        for (int i = 0; i < 3; ++i) x[i] |= (uint32_t)((h >> (3 * b + (2 - i))) & 1u) << b;
+    uint32_t t = x[2] >> 1;
+    for (int i = 2; i > 0; --i) x[i] ^= x[i - 1];
+    x[0] ^= t;
+    for (uint32_t q = 2; q != (1u << bits); q <<= 1) {
+        uint32_t p = q - 1;
+        for (int i = 2; i >= 0; --i) {
+            if (x[i] & q) {
+                x[0] ^= p;
+            } else {
+                uint32_t s = (x[0] ^ x[i]) & p;
+                x[0] ^= s;
+                x[i] ^= s;
+            }
+        }
+    }
+    c[0] = x[0]; c[1] = x[1]; c[2] = x[2];
+}
+
+void oracle_hilbert_row_tokens(int32_t T, int32_t Y, int32_t X, int32_t bs, int32_t* row_token, int64_t n_rows) {
+    int bits = 1;
+    int32_t mx = T > Y ? (T > X ? T : X) : (Y > X ? Y : X);
+    while ((1 << bits) < mx) ++bits;
+    uint64_t cells = 1ull << (3 * bits);
+    int64_t r = 0;
+    (void)bs;
+    for (uint64_t h = 0; h < cells; ++h) {
+        uint32_t c[3];
+        hilbert_cell(h, bits, c);
+        if ((int32_t)c[0] < T && (int32_t)c[1] < Y && (int32_t)c[2] < X)
+            row_token[r++] = (int32_t)(((int64_t)c[0] * Y + c[1]) * X + c[2]);
+    }
+    for (; r < n_rows; ++r) row_token[r] = -1;
+}

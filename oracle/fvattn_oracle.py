@@ -200,6 +200,16 @@ def augment(res: RouteResult, extra: np.ndarray) -> RouteResult:
                        order=res.order, cum_at=res.cum_at, cum_before=res.cum_before, gap=res.gap)
 
 
+def hilbert_row_tokens(T: int, Y: int, X: int, block_tokens: int) -> np.ndarray:
+    """Token at every position of the 3-D Hilbert curve through the grid (-1 on the padding rows)."""
+    n = T * Y * X
+    n_rows = -(-n // block_tokens) * block_tokens
+    out = np.empty(n_rows, dtype=np.int32)
+    lib().oracle_hilbert_row_tokens(ctypes.c_int32(T), ctypes.c_int32(Y), ctypes.c_int32(X),
+                                    ctypes.c_int32(block_tokens), _p(out), ctypes.c_int64(n_rows))
+    return out
+
+
 def sparse_attn(q_r: np.ndarray, k_r: np.ndarray, v_r: np.ndarray, idx: np.ndarray, counts: np.ndarray,
                 g: Grid, sm_scale: float, tiles: np.ndarray | None = None) -> np.ndarray:
     """Masked softmax attention over the retained blocks.

@@ -23,6 +23,7 @@ OK, ERR_INVALID_ARG, ERR_UNSUPPORTED_SHAPE, ERR_WORKSPACE_TOO_SMALL, ERR_CUDA, E
 EXPORTS = (
     "fvattn_num_blocks", "fvattn_block_tokens", "fvattn_padded_tokens", "fvattn_workspace_bytes",
     "fvattn_workspace_init", "fvattn_reorder", "fvattn_inverse_reorder", "fvattn_route",
+    "fvattn_hilbert_row_tokens", "fvattn_reorder_by_table", "fvattn_inverse_reorder_by_table",
     "fvattn_augment", "fvattn_sparse_attn", "fvattn_sparse_attn_simt", "fvattn_sparse_attn_noalloc", "fvattn_tile_order",
     "fvattn_device_status",
     "fvattn_status_string",
@@ -169,6 +170,47 @@ def inverse_reorder(x_r: torch.Tensor, grid: Grid, out: torch.Tensor | None = No
         out = torch.empty(B, grid.tokens, H, d, dtype=torch.bfloat16, device=x_r.device)
     _check(lib().fvattn_inverse_reorder(_ptr(x_r), ctypes.byref(grid.c()), _ptr(out), _layout(out), _stream()),
            "fvattn_inverse_reorder")
+    return out
+
+
+def hilbert_row_tokens(T: int, Y: int, X: int, block_tokens: int) -> torch.Tensor:
+    """Host int32 table: token at every position of the 3-D Hilbert curve through the grid (-1 = padding)."""
+    n = T * Y * X
+    n_rows = -(-n // block_tokens) * block_tokens
+    table = torch.empty(n_rows, dtype=torch.int32)
+    _check(lib().fvattn_hilbert_row_tokens(T, Y, X, block_tokens, ctypes.c_void_p(table.data_ptr()),
+                                           ctypes.c_int64(n_rows)), "fvattn_hilbert_row_tokens")
+    return table
+
+
+def table_grid(n_tokens: int, block_tokens: int) -> Grid:
+    """The 1-D grid under which route / sparse_attn / augment see a table-driven layout."""
+    return Grid(1, 1, n_tokens, 1, 1, block_tokens)
+
+
+def reorder_by_table(x: torch.Tensor, row_token: torch.Tensor, block_tokens: int,
+                     out: torch.Tensor | None = None) -> torch.Tensor:
+    """x [B, N, H, d] bf16 -> [B, H, N_pad, d] with row r holding token row_token[r] (device int32 table)."""
+    _need_cuda(x, row_token)
+    B, N, H, d = x.shape
+    assert row_token.dtype == torch.int32 and row_token.is_contiguous() and x.dtype == torch.bfloat16
+    if out is None:
+        out = torch.empty(B, H, row_token.numel(), d, dtype=torch.bfloat16, device=x.device)
+    _check(lib().fvattn_reorder_by_table(_ptr(x), _layout(x), _ptr(row_token), ctypes.c_int64(N),
+                                         ctypes.c_int32(block_tokens), _ptr(out), _stream()), "fvattn_reorder_by_table")
+    return out
+
+
+def inverse_reorder_by_table(x_r: torch.Tensor, row_token: torch.Tensor, n_tokens: int, block_tokens: int,
+                             out: torch.Tensor | None = None) -> torch.Tensor:
+    _need_cuda(x_r, row_token)
+    B, H, n_pad, d = x_r.shape
+    assert n_pad == row_token.numel() and x_r.is_contiguous()
+    if out is None:
+        out = torch.empty(B, n_tokens, H, d, dtype=torch.bfloat16, device=x_r.device)
+    _check(lib().fvattn_inverse_reorder_by_table(_ptr(x_r), _ptr(row_token), ctypes.c_int64(n_tokens),
+                                                 ctypes.c_int32(block_tokens), _ptr(out), _layout(out), _stream()),
+           "fvattn_inverse_reorder_by_table")
     return out
 
 

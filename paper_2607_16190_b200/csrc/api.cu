@@ -68,14 +68,42 @@ fvattn_status_t fvattn_reorder(const void* src, fvattn_tok_layout_t lay, const f
                                fvattn_stream_t stream) {
     fvattn_status_t st = check_layout(lay, src, dst_r, grid);
     if (st != FVATTN_OK) return st;
-    return launch_reorder(src, lay, make_dims(*grid), dst_r, (cudaStream_t)stream);
+    return launch_reorder(src, lay, make_dims(*grid), dst_r, nullptr, (cudaStream_t)stream);
 }
 
 fvattn_status_t fvattn_inverse_reorder(const void* src_r, const fvattn_grid_t* grid, void* dst,
                                        fvattn_tok_layout_t lay, fvattn_stream_t stream) {
     fvattn_status_t st = check_layout(lay, dst, src_r, grid);
     if (st != FVATTN_OK) return st;
-    return launch_inverse_reorder(src_r, make_dims(*grid), dst, lay, (cudaStream_t)stream);
+    return launch_inverse_reorder(src_r, make_dims(*grid), dst, lay, nullptr, (cudaStream_t)stream);
+}
+
+// A table-driven layout is the 1-D grid of n_rows / Bs blocks: (T, Y, X) = (1, 1, n_tokens), tile (1, 1, Bs).
+static fvattn_status_t table_grid(int64_t n_tokens, int32_t block_tokens, const int32_t* row_token,
+                                  fvattn_grid_t* g) {
+    if (!row_token || n_tokens <= 0 || n_tokens > 0x7fffffffLL || block_tokens <= 0) return FVATTN_ERR_INVALID_ARG;
+    *g = fvattn_grid_t{1, 1, (int32_t)n_tokens, 1, 1, block_tokens};
+    return FVATTN_OK;
+}
+
+fvattn_status_t fvattn_reorder_by_table(const void* src, fvattn_tok_layout_t lay, const int32_t* row_token,
+                                        int64_t n_tokens, int32_t block_tokens, void* dst_r,
+                                        fvattn_stream_t stream) {
+    fvattn_grid_t g;
+    fvattn_status_t st = table_grid(n_tokens, block_tokens, row_token, &g);
+    if (st == FVATTN_OK) st = check_layout(lay, src, dst_r, &g);
+    if (st != FVATTN_OK) return st;
+    return launch_reorder(src, lay, make_dims(g), dst_r, row_token, (cudaStream_t)stream);
+}
+
+fvattn_status_t fvattn_inverse_reorder_by_table(const void* src_r, const int32_t* row_token, int64_t n_tokens,
+                                                int32_t block_tokens, void* dst, fvattn_tok_layout_t lay,
+                                                fvattn_stream_t stream) {
+    fvattn_grid_t g;
+    fvattn_status_t st = table_grid(n_tokens, block_tokens, row_token, &g);
+    if (st == FVATTN_OK) st = check_layout(lay, dst, src_r, &g);
+    if (st != FVATTN_OK) return st;
+    return launch_inverse_reorder(src_r, make_dims(g), dst, lay, row_token, (cudaStream_t)stream);
 }
 
 fvattn_status_t fvattn_route(const void* q_r, const void* k_r, int32_t B, int32_t H, int32_t d,

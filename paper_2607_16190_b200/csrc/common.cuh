@@ -133,9 +133,9 @@ inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_
 
 // ---- kernel launchers implemented by the other translation units -------------------------
 fvattn_status_t launch_reorder(const void* src, const fvattn_tok_layout_t& lay, const GridDims& m, void* dst_r,
-                               cudaStream_t s);
+                               const int32_t* row_token, cudaStream_t s);
 fvattn_status_t launch_inverse_reorder(const void* src_r, const GridDims& m, void* dst,
-                                       const fvattn_tok_layout_t& lay, cudaStream_t s);
+                                       const fvattn_tok_layout_t& lay, const int32_t* row_token, cudaStream_t s);
 fvattn_status_t launch_route(const void* q_r, const void* k_r, int64_t BH, int d, const GridDims& m, float p,
                              int k_floor, float sm_scale, uint32_t* mask_bits, int32_t* counts, uint16_t* idx,
                              float* head_load, void* workspace, cudaStream_t s);

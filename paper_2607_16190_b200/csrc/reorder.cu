@@ -16,7 +16,8 @@ constexpr int kMaxBs = 128;
 template <bool kInverse, int VPR /* 16-byte vectors per row: d / 8 */>
 __global__ void __launch_bounds__(kReorderThreads)
 reorder_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, GridDims m, int H,
-               int64_t sb, int64_t sn, int64_t sh /* strides of the token layout in 16-byte vectors */) {
+               int64_t sb, int64_t sn, int64_t sh /* strides of the token layout in 16-byte vectors */,
+               const int32_t* __restrict__ row_token /* NULL: 3-D tiles; else token of each tiled row, -1 = padding */) {
     constexpr int kItems = kHeadChunk * VPR;                   // (head, vector) pairs per row
     constexpr int kRowsPerPass = kReorderThreads / kItems;     // 2 for d = 128, 4 for d = 64
     __shared__ int64_t tok[kMaxBs];                            // token of each row, -1 for padding
@@ -26,8 +27,13 @@ reorder_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, GridDims 
     const int hc = min(kHeadChunk, H - h0);
     const int b = blockIdx.z;
     for (int o = threadIdx.x; o < m.bs; o += kReorderThreads) {
-        int64_t token;
-        tok[o] = row_to_token(m, blk, o, &token) ? token : -1;
+        if (row_token) {
+            const int64_t t = row_token[(int64_t)blk * m.bs + o];
+            tok[o] = (t >= 0 && t < m.n) ? t : -1;             // anything outside the token range is padding
+        } else {
+            int64_t token;
+            tok[o] = row_to_token(m, blk, o, &token) ? token : -1;
+        }
     }
     __syncthreads();
 
@@ -64,27 +70,27 @@ reorder_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, GridDims 
 
 template <bool kInverse>
 static fvattn_status_t launch_any(const void* src, void* dst, const fvattn_tok_layout_t& lay, const GridDims& m,
-                                  cudaStream_t s) {
+                                  const int32_t* row_token, cudaStream_t s) {
     if (m.bs > kMaxBs) return FVATTN_ERR_UNSUPPORTED_SHAPE;
     dim3 grid((unsigned)m.nb, (unsigned)((lay.H + kHeadChunk - 1) / kHeadChunk), (unsigned)lay.B);
     const int64_t sb = lay.stride_b / 8, sn = lay.stride_n / 8, sh = lay.stride_h / 8;
     if (lay.d == 128)
-        reorder_kernel<kInverse, 16><<<grid, kReorderThreads, 0, s>>>((const uint4*)src, (uint4*)dst, m, lay.H, sb, sn, sh);
+        reorder_kernel<kInverse, 16><<<grid, kReorderThreads, 0, s>>>((const uint4*)src, (uint4*)dst, m, lay.H, sb, sn, sh, row_token);
     else if (lay.d == 64)
-        reorder_kernel<kInverse, 8><<<grid, kReorderThreads, 0, s>>>((const uint4*)src, (uint4*)dst, m, lay.H, sb, sn, sh);
+        reorder_kernel<kInverse, 8><<<grid, kReorderThreads, 0, s>>>((const uint4*)src, (uint4*)dst, m, lay.H, sb, sn, sh, row_token);
     else
         return FVATTN_ERR_UNSUPPORTED_SHAPE;
     return launch_status();
 }
 
 fvattn_status_t launch_reorder(const void* src, const fvattn_tok_layout_t& lay, const GridDims& m, void* dst_r,
-                               cudaStream_t s) {
-    return launch_any<false>(src, dst_r, lay, m, s);
+                               const int32_t* row_token, cudaStream_t s) {
+    return launch_any<false>(src, dst_r, lay, m, row_token, s);
 }
 
 fvattn_status_t launch_inverse_reorder(const void* src_r, const GridDims& m, void* dst,
-                                       const fvattn_tok_layout_t& lay, cudaStream_t s) {
-    return launch_any<true>(src_r, dst, lay, m, s);
+                                       const fvattn_tok_layout_t& lay, const int32_t* row_token, cudaStream_t s) {
+    return launch_any<true>(src_r, dst, lay, m, row_token, s);
 }
 
 } // namespace fvattn

@@ -1,0 +1,71 @@
+"""Hilbert-curve block organisation (Sec. 3.1): the library's table (coordinates -> curve index, then a
+sort) against the oracle's walk (curve index -> coordinates), and the table-driven reorder and the rest
+of the path on that layout against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import fvattn_oracle as O
+from paper_2607_16190_b200 import binding as fv
+from paper_2607_16190_b200 import synth
+
+
+@pytest.mark.parametrize("shape,bs", [((4, 8, 8), 64), ((3, 5, 7), 64), ((8, 16, 16), 128), ((21, 30, 52), 128),
+                                      ((21, 45, 80), 128)])
+def test_library_table_equals_oracle_walk(shape, bs):
+    np.testing.assert_array_equal(fv.hilbert_row_tokens(*shape, bs).numpy(), O.hilbert_row_tokens(*shape, bs))
+
+
+def test_table_argument_errors():
+    import ctypes
+    buf = (ctypes.c_int32 * 64)()
+    L = fv.lib()
+    assert L.fvattn_hilbert_row_tokens(2, 2, 2, 8, buf, ctypes.c_int64(16)) == fv.ERR_INVALID_ARG   # wrong n_rows
+    assert L.fvattn_hilbert_row_tokens(0, 2, 2, 8, buf, ctypes.c_int64(8)) == fv.ERR_INVALID_ARG
+    assert L.fvattn_hilbert_row_tokens(2, 2, 2, 8, buf, ctypes.c_int64(8)) == fv.OK
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("name", ["small", "wan480p"])
+def test_hilbert_layout_reorder_route_attention_match_oracle(name):
+    cfg = synth.CONFIGS[name]
+    T, Y, X = cfg.grid
+    bs, n = cfg.block_tokens, cfg.tokens
+    q, k, v, _ = synth.make_qkv(cfg, "cuda")
+    table = fv.hilbert_row_tokens(T, Y, X, bs)
+    tab_np = table.numpy()
+    tab_dev = table.cuda()
+    # reorder: row r of every head holds token table[r]; padding rows are zero; the inverse restores
+    q_r, k_r, v_r = (fv.reorder_by_table(t, tab_dev, bs) for t in (q, k, v))
+    qh = synth.bf16_bits(q)[0]                                        # [N, H, d]
+    want = np.zeros((cfg.H, tab_np.size, cfg.d), dtype=np.uint16)
+    want[:, tab_np >= 0] = qh[tab_np[tab_np >= 0]].transpose(1, 0, 2)
+    np.testing.assert_array_equal(synth.bf16_bits(q_r)[0], want)
+    assert torch.equal(fv.inverse_reorder_by_table(q_r, tab_dev, n, bs), q)
+    # route + attention see the layout as a 1-D grid of consecutive blocks
+    g = fv.table_grid(n, bs)
+    og = O.Grid(1, 1, n, 1, 1, bs)
+    ws = fv.make_workspace(g, 1, cfg.H, cfg.d)
+    res = fv.route(q_r, k_r, g, cfg.p, cfg.k_floor, cfg.sm_scale, ws)
+    qb, kb, vb = (synth.bf16_bits(t)[0] for t in (q_r, k_r, v_r))
+    res_o = O.route(qb, kb, og, cfg.p, cfg.k_floor, cfg.sm_scale)
+    diff = (res.mask_bits[0].cpu().numpy() != res_o.mask_bits).any(-1)
+    near = (np.abs(res_o.cum_at - cfg.p) < 1e-5) | (np.abs(res_o.cum_before - cfg.p) < 1e-5)
+    assert not (diff & ~near & ~(res_o.gap < 1e-6)).any()
+    idx = torch.from_numpy(res_o.idx).cuda()[None]
+    counts = torch.from_numpy(res_o.counts).cuda()[None]
+    o_r = fv.sparse_attn(q_r, k_r, v_r, idx, counts, g, cfg.sm_scale, ws)
+    assert fv.device_status(ws) == fv.OK
+    nb = g.num_blocks
+    rng = np.random.default_rng(0)
+    tiles = np.unique(np.concatenate([[nb - 1, cfg.H * nb - 1], rng.integers(0, cfg.H * nb, 10)])).astype(np.int64)
+    want_o = O.sparse_attn(qb, kb, vb, res_o.idx, res_o.counts, og, cfg.sm_scale, tiles=tiles)
+    got = o_r[0].reshape(cfg.H * nb, bs, cfg.d)[torch.from_numpy(tiles).cuda()].float().cpu().numpy()
+    err = np.abs(got - want_o)
+    assert err.max() <= 1e-2 and err.mean() <= 1e-3
+    # density at equal p: curve blocks against 3-D tiles on the same inputs
+    gt, ogt = fv.Grid(*cfg.grid, *cfg.tile), O.Grid(*cfg.grid, *cfg.tile)
+    res_t = O.route(*(O.reorder(synth.bf16_bits(t), ogt)[0] for t in (q, k)), ogt, cfg.p, cfg.k_floor, cfg.sm_scale)
+    print(f"\n[{name}] density at p={cfg.p}: Hilbert blocks {res_o.counts.mean() / nb:.4f} ({nb} blocks), "
+          f"3-D tiles {res_t.counts.mean() / gt.num_blocks:.4f} ({gt.num_blocks} blocks); mask rows differing {int(diff.sum())}; "
+          f"attention max-abs {err.max():.2e}")

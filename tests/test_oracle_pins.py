@@ -258,6 +258,49 @@ def test_hand_worked_rows():
             assert res.idx[0, i, :len(kept)].tolist() == kept, (case, i)
 
 
+# ---------------------------------------------------------------- Hilbert organisation (Sec. 3.1)
+def test_hilbert_walk_on_a_full_cube_is_a_unit_step_octree_curve():
+    """What makes a curve a Hilbert curve: it visits every cell once, moves one cell at a time, and
+    every aligned sub-cube of side 2^j is traversed in one contiguous run of 8^j positions."""
+    for side in (2, 4, 8, 16):
+        tab = O.hilbert_row_tokens(side, side, side, 8)
+        n = side ** 3
+        assert sorted(tab.tolist()) == list(range(n))
+        assert tab[0] == 0                                          # starts at the origin
+        t, y, x = np.unravel_index(tab, (side, side, side))
+        step = np.abs(np.diff(t)) + np.abs(np.diff(y)) + np.abs(np.diff(x))
+        assert (step == 1).all()
+        j = 2
+        while j < side:
+            run = j ** 3
+            for r0 in range(0, n, run):
+                tt, yy, xx = t[r0:r0 + run], y[r0:r0 + run], x[r0:r0 + run]
+                assert tt.max() - tt.min() == j - 1 and yy.max() - yy.min() == j - 1 and xx.max() - xx.min() == j - 1
+                assert tt.min() % j == 0 and yy.min() % j == 0 and xx.min() % j == 0
+            j *= 2
+
+
+@pytest.mark.parametrize("shape,bs", [((4, 8, 8), 64), ((3, 5, 7), 8), ((21, 45, 80), 128)])
+def test_hilbert_rows_on_a_ragged_grid(shape, bs):
+    T, Y, X = shape
+    n = T * Y * X
+    tab = O.hilbert_row_tokens(T, Y, X, bs)
+    assert tab.size == -(-n // bs) * bs and (tab[n:] == -1).all()
+    assert sorted(tab[:n].tolist()) == list(range(n))               # bijection onto the tokens
+    # the order is the cube's curve order restricted to the grid: positions in the full cube increase
+    side = 1
+    while side < max(shape):
+        side *= 2
+    cube = O.hilbert_row_tokens(side, side, side, 1)
+    pos_in_cube = np.empty(side ** 3, dtype=np.int64)
+    pos_in_cube[cube] = np.arange(side ** 3)
+    t, y, x = np.unravel_index(tab[:n], shape)
+    assert (np.diff(pos_in_cube[(t * side + y) * side + x]) > 0).all()
+    # locality: most consecutive tokens are neighbours, and blocks are spatially compact
+    step = np.abs(np.diff(t)) + np.abs(np.diff(y)) + np.abs(np.diff(x))
+    assert (step == 1).mean() > 0.9
+
+
 # ---------------------------------------------------------------- augmentation (Sec. 3.3)
 def test_augmentation_appends_the_next_ranks_and_only_grows_the_mask():
     cfg, g, q_r, k_r, _ = _routing_inputs("small")
