@@ -5,8 +5,8 @@
 //   warp 0        producer: pops (head, query-block) tiles from the heaviest-first queue, TMA-loads
 //                 Q once per tile and the retained K tiles by index into a 3-deep ring
 //   warp 2        second producer: the retained V tiles into their own 3-deep ring
-//   warp 1        MMA issuer (one thread): S = Q K^T and O += P V as tcgen05 MMAs, accumulators in
-//                 tensor memory
+//   warps 1, 3    MMA issuers (one thread each): warp 1 issues S = Q K^T, warp 3 issues O += P V, as
+//                 tcgen05 MMAs with the accumulators in tensor memory
 //   warps 4-7     softmax of the even retained blocks  (stream 0)
 //   warps 8-11    softmax of the odd retained blocks   (stream 1)
 // The retained blocks of a tile alternate between two independent streams, each with its own
@@ -53,7 +53,7 @@ struct __align__(1024) Smem {
     unsigned char v[VS][kTileBytes];
     float ml[2][2][BS];                             // [stream][m, l][row]
     unsigned long long q_full, q_empty, k_full[KS], k_empty[KS], v_full[VS], v_empty[VS];
-    unsigned long long s_full[2], p_full[2], o_full, o_free, ml_ready, ml_done, tile_full[TS], tile_empty[TS];
+    unsigned long long s_full[2], p_full[2], pv_done[2], o_full, o_free, ml_ready, ml_done, tile_full[TS], tile_empty[TS];
     int tile_id[TS];
     int tile_cnt[TS];
     uint32_t tmem_base;
@@ -129,12 +129,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         mbar_init(smem_u32(&sm.q_empty), 1);
         for (int s = 0; s < KS; ++s) { mbar_init(smem_u32(&sm.k_full[s]), 1); mbar_init(smem_u32(&sm.k_empty[s]), 1); }
         for (int s = 0; s < VS; ++s) { mbar_init(smem_u32(&sm.v_full[s]), 1); mbar_init(smem_u32(&sm.v_empty[s]), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&sm.s_full[a]), 1); mbar_init(smem_u32(&sm.p_full[a]), 4); }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(smem_u32(&sm.s_full[a]), 1);
+            mbar_init(smem_u32(&sm.p_full[a]), 4);
+            mbar_init(smem_u32(&sm.pv_done[a]), 1);
+        }
         mbar_init(smem_u32(&sm.o_full), 1);
         mbar_init(smem_u32(&sm.o_free), 8);
         mbar_init(smem_u32(&sm.ml_ready), 8);
         mbar_init(smem_u32(&sm.ml_done), 8);
-        for (int s = 0; s < TS; ++s) { mbar_init(smem_u32(&sm.tile_full[s]), 1); mbar_init(smem_u32(&sm.tile_empty[s]), 10); }
+        for (int s = 0; s < TS; ++s) { mbar_init(smem_u32(&sm.tile_full[s]), 1); mbar_init(smem_u32(&sm.tile_empty[s]), 11); }
         sm.abort_flag = 0;
         fence_barrier_init();
         prefetch_tensormap(&map_q);
@@ -267,38 +271,23 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
             }
             failed = !ok;
-        } else if (warp == 1 && lane == 0) {
-            // ======================= MMA issuer (one thread) ===========================================
+        } else if ((warp == 1 || warp == 3) && lane == 0) {
+            // ======================= MMA issuers: one thread for S = Q K^T, one for O += P V =============
+            // Two threads on two schedulers halve the serial time per block that a single issuer spends on
+            // barrier polls, commits and MMA instructions.  The only ordering the two need between them is
+            // that QK(t + 2) must not overwrite the S/P columns of stream a before PV(t) has read P: the
+            // QK thread waits for the completion of PV(t) (pv_done, a commit by the PV thread).
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, true);
-            uint32_t n = 0, kn = 0, vn = 0, qn = 0, pn[2] = {0, 0};
-            bool ok = true;
             // descriptor words that never change: high word (stride 1024 B, version, 128-byte swizzle);
             // low word = (address >> 4) | (leading offset >> 4) << 16, advanced by adding (bytes >> 4)
             const uint32_t desc_hi = (uint32_t)(make_smem_desc_sw128(0, 16, 1024) >> 32);
             const uint32_t q_lo = (uint32_t)make_smem_desc_sw128(smem_u32(sm.q), 16, 1024);
             const uint32_t k_lo0 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.k[0]), 16, 1024);
             const uint32_t v_lo0 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.v[0]), kHalfBytes, 1024);
-
-            auto issue_pv = [&](int u) {
-                const int b = u & 1;
-                ok = ok && mbar_wait(smem_u32(&sm.p_full[b]), pn[b] & 1u, abort_flag);
-                ++pn[b];
-                const uint32_t vs = vn % VS;
-                ok = ok && mbar_wait(smem_u32(&sm.v_full[vs]), (vn / VS) & 1u, abort_flag);
-                if (u == 0) ok = ok && mbar_wait(smem_u32(&sm.o_free), (qn & 1u) ^ 1u, abort_flag);
-                if (ok) {
-                    tc_fence_after();
-                    const uint32_t vlo = v_lo0 + vs * (kTileBytes >> 4);
-                    const uint32_t tOb = tmem + kColO + 128u * b, tPb = tmem + kColS + 128u * b;
-#pragma unroll
-                    for (int ks = 0; ks < BS / 16; ++ks)
-                        umma_ts(tOb, tPb + ks * 8, ((uint64_t)desc_hi << 32) | (vlo + (uint32_t)ks * (2048u >> 4)), idesc_pv,
-                                (u >= 2 || ks > 0) ? 1u : 0u);
-                    umma_commit(smem_u32(&sm.v_empty[vs]));
-                }
-                ++vn;
-            };
+            uint32_t n = 0, ring = 0, qn = 0, cnt0 = 0, cnt1 = 0;   // cnt: blocks of each stream so far
+            bool ok = true;
+            const bool is_qk = warp == 1;
 
             while (ok) {
                 const uint32_t slot = n % TS;
@@ -310,29 +299,54 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 ++n;
                 if (tile < 0) break;
                 if (c == 0) continue;
-                ok = mbar_wait(smem_u32(&sm.q_full), qn & 1u, abort_flag);
-                for (int t = 0; t < c && ok; ++t) {
-                    const int a = t & 1;
-                    const uint32_t ks_ = kn % KS;
-                    ok = mbar_wait(smem_u32(&sm.k_full[ks_]), (kn / KS) & 1u, abort_flag);
-                    if (!ok) break;
-                    tc_fence_after();
-                    const uint32_t klo = k_lo0 + ks_ * (kTileBytes >> 4);
-                    const uint32_t tSa = tmem + kColS + 128u * a;
+                if (is_qk) {
+                    ok = mbar_wait(smem_u32(&sm.q_full), qn & 1u, abort_flag);
+                    for (int t = 0; t < c && ok; ++t) {
+                        const int a = t & 1;
+                        uint32_t& cnt = a ? cnt1 : cnt0;
+                        const uint32_t st = ring % KS, ph = (ring / KS) & 1u;
+                        // the previous block of this stream (possibly of the previous tile) must have been read by its PV
+                        if (cnt > 0) ok = mbar_wait(smem_u32(&sm.pv_done[a]), (cnt - 1u) & 1u, abort_flag);
+                        ok = ok && mbar_wait(smem_u32(&sm.k_full[st]), ph, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t klo = k_lo0 + st * (kTileBytes >> 4);
+                        const uint32_t tSa = tmem + kColS + 128u * a;
 #pragma unroll
-                    for (int ks = 0; ks < D / 16; ++ks) {
-                        const uint32_t off16 = ((uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u) >> 4;
-                        umma_ss(tSa, ((uint64_t)desc_hi << 32) | (q_lo + off16), ((uint64_t)desc_hi << 32) | (klo + off16),
-                                idesc_qk, ks > 0 ? 1u : 0u);
+                        for (int ks = 0; ks < D / 16; ++ks) {
+                            const uint32_t off16 = ((uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u) >> 4;
+                            umma_ss(tSa, ((uint64_t)desc_hi << 32) | (q_lo + off16), ((uint64_t)desc_hi << 32) | (klo + off16),
+                                    idesc_qk, ks > 0 ? 1u : 0u);
+                        }
+                        umma_commit(smem_u32(&sm.k_empty[st]));
+                        if (t == c - 1) umma_commit(smem_u32(&sm.q_empty));
+                        umma_commit(smem_u32(&sm.s_full[a]));
+                        ++cnt;
+                        ++ring;
                     }
-                    umma_commit(smem_u32(&sm.k_empty[ks_]));
-                    ++kn;
-                    if (t == c - 1) umma_commit(smem_u32(&sm.q_empty));
-                    umma_commit(smem_u32(&sm.s_full[a]));
-                    if (t >= 1) issue_pv(t - 1);
+                } else {
+                    for (int t = 0; t < c && ok; ++t) {
+                        const int b = t & 1;
+                        uint32_t& cnt = b ? cnt1 : cnt0;
+                        const uint32_t st = ring % VS, ph = (ring / VS) & 1u;
+                        ok = mbar_wait(smem_u32(&sm.p_full[b]), cnt & 1u, abort_flag) &&
+                             mbar_wait(smem_u32(&sm.v_full[st]), ph, abort_flag);
+                        if (ok && t == 0) ok = mbar_wait(smem_u32(&sm.o_free), (qn & 1u) ^ 1u, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
+                        const uint32_t vlo = v_lo0 + st * (kTileBytes >> 4);
+                        const uint32_t tOb = tmem + kColO + 128u * b, tPb = tmem + kColS + 128u * b;
+#pragma unroll
+                        for (int ks = 0; ks < BS / 16; ++ks)
+                            umma_ts(tOb, tPb + ks * 8, ((uint64_t)desc_hi << 32) | (vlo + (uint32_t)ks * (2048u >> 4)), idesc_pv,
+                                    (t >= 2 || ks > 0) ? 1u : 0u);
+                        umma_commit(smem_u32(&sm.v_empty[st]));
+                        umma_commit(smem_u32(&sm.pv_done[b]));
+                        ++cnt;
+                        ++ring;
+                    }
+                    if (ok) umma_commit(smem_u32(&sm.o_full));   // every PV done implies every QK done
                 }
-                if (ok) issue_pv(c - 1);
-                if (ok) umma_commit(smem_u32(&sm.o_full));
                 ++qn;
             }
             failed = !ok;
