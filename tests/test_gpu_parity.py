@@ -170,6 +170,42 @@ def test_route_more_than_1024_blocks_uses_the_sorting_kernel():
               f"density {res_o.counts.mean() / 1280:.4f}")
 
 
+def test_route_exactly_1024_blocks_uses_the_widest_warp_kernel():
+    """nb = 1024: 32 entries per lane in the warp selection kernel."""
+    cfg = synth.Config("nb1024", 1, 64, (4, 128, 128), (1, 8, 8), 0.9, 2, 16, "loguniform", seed=41)
+    g, og = grids(cfg)
+    assert g.num_blocks == 1024
+    q, k, _, _ = synth.make_qkv(cfg, "cuda")
+    q_r, k_r = fv.reorder(q, g), fv.reorder(k, g)
+    ws = fv.make_workspace(g, 1, cfg.H, cfg.d)
+    res = fv.route(q_r, k_r, g, cfg.p, cfg.k_floor, cfg.sm_scale, ws)
+    assert fv.device_status(ws) == fv.OK
+    res_o = O.route(synth.bf16_bits(q_r)[0], synth.bf16_bits(k_r)[0], og, cfg.p, cfg.k_floor, cfg.sm_scale)
+    ndiff, nnear, ntie = compare_masks(res, res_o, cfg.p)
+    print(f"\n[nb=1024] differing {ndiff}, near-threshold {nnear}, near-tie {ntie}")
+
+
+@pytest.mark.parametrize("tile,d", [((1, 8, 8), 128), ((2, 8, 8), 64)])
+def test_attention_mixed_block_and_head_sizes(tile, d):
+    """Bs = 64 with d = 128 and Bs = 128 with d = 64: the CUDA-core kernel's other two instantiations."""
+    cfg = synth.Config("mixed", 3, d, (4, 16, 16), tile, 0.8, 2, 16, "loguniform", seed=51)
+    g, og = grids(cfg)
+    q, k, v, _ = synth.make_qkv(cfg, "cuda")
+    q_r, k_r, v_r = (fv.reorder(t, g) for t in (q, k, v))
+    qb, kb, vb = (synth.bf16_bits(t)[0] for t in (q_r, k_r, v_r))
+    ws = fv.make_workspace(g, 1, cfg.H, cfg.d)
+    res = fv.route(q_r, k_r, g, cfg.p, cfg.k_floor, cfg.sm_scale, ws)
+    res_o = O.route(qb, kb, og, cfg.p, cfg.k_floor, cfg.sm_scale)
+    compare_masks(res, res_o, cfg.p)
+    idx = torch.from_numpy(res_o.idx).cuda()[None]
+    counts = torch.from_numpy(res_o.counts).cuda()[None]
+    o_r = fv.sparse_attn(q_r, k_r, v_r, idx, counts, g, cfg.sm_scale, ws)
+    assert fv.device_status(ws) == fv.OK
+    want = O.sparse_attn(qb, kb, vb, res_o.idx, res_o.counts, og, cfg.sm_scale)
+    mx, mean = attn_errors(o_r[0].float().cpu().numpy(), want)
+    assert mx <= MAX_ABS and mean <= MEAN_ABS
+
+
 def test_batch_of_two_routes_and_attends_like_two_single_batches():
     """B = 2: (batch, head) pairs are independent; results equal the per-batch calls bit for bit."""
     cfg = synth.CONFIGS["small"]
