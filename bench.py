@@ -274,25 +274,30 @@ def run_ours(args):
     ms_per_step = total_ms / args.steps
     value = flops_all / (ms_per_step * 1e-3) / 1e12
 
-    # ---- e2e: pinned host inputs, H2D + path + D2H of the output inside the timed region
+    # ---- e2e: pinned host inputs; every step uploads Q, K, V, runs the path and downloads the output,
+    # all inside the timed region.  HostPipeline overlaps the copies of step i + 1 with the kernels of
+    # step i (double-buffered device inputs / outputs), which is how a caller feeding layers from the
+    # host would drive the library.
     hq, hk, hv = (t.cpu().pin_memory() for t in (q, k, v))
-    hout = torch.empty_like(hq).pin_memory()
-    dq, dk, dv = (torch.empty_like(t) for t in (q, k, v))
+    hout = [torch.empty_like(hq).pin_memory() for _ in range(2)]
+    pipe = fv.HostPipeline(layer)
 
-    def e2e_step():
-        dq.copy_(hq, non_blocking=True); dk.copy_(hk, non_blocking=True); dv.copy_(hv, non_blocking=True)
-        out = layer(dq, dk, dv)
-        hout.copy_(out, non_blocking=True)
+    def e2e_run(steps):
+        for i in range(steps):
+            pipe.submit(hq, hk, hv, hout[i & 1])
+        pipe.drain()
 
-    e2e_step()
+    e2e_run(2)
+    torch.cuda.synchronize()
     if world > 1:
         dist.barrier()
-    e2e_steps = max(2, min(args.steps, 5))
-    e2e_ms = time_steps(e2e_step, e2e_steps, torch) / e2e_steps
+    e2e_steps = max(4, min(args.steps, 10))
+    e2e_ms = time_steps(lambda: e2e_run(e2e_steps), 1, torch) / e2e_steps
     e2e_ms = replicas.max_over_ranks(e2e_ms, world, dev)
     e2e = {"value": flops_all / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": e2e_ms,
-           "h2d_bytes_per_step": 3 * hq.numel() * 2, "d2h_bytes_per_step": hout.numel() * 2}
-    del hq, hk, hv, hout, dq, dk, dv
+           "h2d_bytes_per_step": 3 * hq.numel() * 2, "d2h_bytes_per_step": hout[0].numel() * 2,
+           "pipelined": "copies of step i+1 overlap the kernels of step i (3 streams, double-buffered)"}
+    del hq, hk, hv, hout, pipe
 
     if rank != 0:
         if world > 1:

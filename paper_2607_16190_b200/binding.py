@@ -343,3 +343,58 @@ class SparseAttentionLayer:
         sparse_attn(self.q_r, self.k_r, self.v_r, self.routing.idx, self.routing.counts, g, self.sm_scale,
                     self.workspace, self.o_r)
         return inverse_reorder(self.o_r, g, self.out)
+
+
+class HostPipeline:
+    """Runs a SparseAttentionLayer on inputs that live in pinned HOST memory, one call per layer
+    invocation, with the copies of consecutive calls overlapped with the kernels: the inputs of call
+    i + 1 are uploaded on a copy stream while call i computes, and the output of call i goes back on a
+    third stream.  Device inputs and outputs are double-buffered; nothing is allocated per call."""
+
+    def __init__(self, layer: SparseAttentionLayer):
+        self.layer = layer
+        dev = layer.q_r.device
+        shape = (layer.B, layer.grid.tokens, layer.H, layer.d)
+        self.dq, self.dk, self.dv, self.dout = ([torch.empty(shape, dtype=torch.bfloat16, device=dev) for _ in range(2)]
+                                                for _ in range(4))
+        self.s_in, self.s_comp, self.s_out = (torch.cuda.Stream(device=dev) for _ in range(3))
+        self.ev_in = [torch.cuda.Event() for _ in range(2)]
+        self.ev_comp = [torch.cuda.Event() for _ in range(2)]
+        self.ev_out = [torch.cuda.Event() for _ in range(2)]
+        self.calls = 0
+
+    def submit(self, hq: torch.Tensor, hk: torch.Tensor, hv: torch.Tensor, hout: torch.Tensor) -> None:
+        """Enqueue one layer: hq, hk, hv, hout are pinned host tensors [B, N, H, d] bf16.  Returns at once;
+        `hout` is complete after `drain()` (or once two more calls have been submitted and synchronised)."""
+        L, b = self.layer, self.calls & 1
+        cur = torch.cuda.current_stream()
+        if self.calls < 2:                      # the first use of each buffer follows the caller's stream
+            self.s_in.wait_stream(cur); self.s_comp.wait_stream(cur); self.s_out.wait_stream(cur)
+        with torch.cuda.stream(self.s_in):
+            if self.calls >= 2:
+                self.s_in.wait_event(self.ev_comp[b])          # the kernels that read this input buffer are done
+            self.dq[b].copy_(hq, non_blocking=True)
+            self.dk[b].copy_(hk, non_blocking=True)
+            self.dv[b].copy_(hv, non_blocking=True)
+            self.ev_in[b].record(self.s_in)
+        with torch.cuda.stream(self.s_comp):
+            self.s_comp.wait_event(self.ev_in[b])
+            if self.calls >= 2:
+                self.s_comp.wait_event(self.ev_out[b])         # the download of this output buffer is done
+            g = L.grid
+            reorder(self.dq[b], g, L.q_r); reorder(self.dk[b], g, L.k_r); reorder(self.dv[b], g, L.v_r)
+            route(L.q_r, L.k_r, g, L.p, L.k_floor, L.sm_scale, L.workspace, L.routing)
+            sparse_attn(L.q_r, L.k_r, L.v_r, L.routing.idx, L.routing.counts, g, L.sm_scale, L.workspace, L.o_r)
+            inverse_reorder(L.o_r, g, self.dout[b])
+            self.ev_comp[b].record(self.s_comp)
+        with torch.cuda.stream(self.s_out):
+            self.s_out.wait_event(self.ev_comp[b])
+            hout.copy_(self.dout[b], non_blocking=True)
+            self.ev_out[b].record(self.s_out)
+        self.calls += 1
+
+    def drain(self) -> None:
+        """Make the caller's current stream wait for everything submitted so far."""
+        cur = torch.cuda.current_stream()
+        for s in (self.s_in, self.s_comp, self.s_out):
+            cur.wait_stream(s)

@@ -433,3 +433,23 @@ def test_whole_layer_matches_oracle_pipeline(name):
     want = want_r[:, O.permutation(og), :].transpose(1, 0, 2)          # [N, H, d]
     mx, mean = attn_errors(out[0].float().cpu().numpy(), want)
     assert mx <= MAX_ABS and mean <= MEAN_ABS
+
+
+def test_host_pipeline_returns_what_the_layer_returns():
+    """Inputs in pinned host memory, copies overlapped with the kernels over several calls."""
+    c = case("small")
+    cfg, g = c["cfg"], c["g"]
+    layer = fv.SparseAttentionLayer(g, 1, cfg.H, cfg.d, cfg.p, cfg.k_floor)
+    want = layer(c["q"], c["k"], c["v"]).clone()
+    other = synth.make_qkv(cfg.with_(seed=99), "cuda")[:3]
+    want_other = layer(*other).clone()
+    host = [tuple(t.cpu().pin_memory() for t in trio) for trio in ((c["q"], c["k"], c["v"]), other)]
+    outs = [torch.empty_like(host[0][0]).pin_memory() for _ in range(5)]
+    pipe = fv.HostPipeline(layer)
+    for i in range(5):
+        pipe.submit(*host[i & 1], outs[i])
+    pipe.drain()
+    torch.cuda.synchronize()
+    assert fv.device_status(layer.workspace) == fv.OK
+    for i in range(5):
+        assert torch.equal(outs[i], (want if i % 2 == 0 else want_other).cpu())
