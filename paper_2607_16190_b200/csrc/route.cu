@@ -158,113 +158,144 @@ pool_kernel(const uint4* __restrict__ q_r, const uint4* __restrict__ k_r, __nv_b
 }
 
 // ----------------------------------------------------------------------------------- scores
-// One CTA per 128 x 128 tile of one head's score matrix.  The six operand tiles (three parts of
-// the 128 query-block means, three of the 128 key-block means) are TMA-loaded with the 128-byte
-// swizzle (rows past nb are zero-filled by the copy engine), one thread issues the 6 x d/16
-// tcgen05 MMAs, and the four warps read the fp32 accumulator from tensor memory, scale it and
-// store their rows.  Small products are accumulated first.
+// Persistent CTAs, each looping over 128 x 128 tiles of the per-head score matrices.  The six
+// operand tiles of a score tile (three parts of 128 query-block means, three of 128 key-block
+// means) are TMA-loaded with the 128-byte swizzle (rows past nb are zero-filled by the copy
+// engine); one thread of warp 4 issues the copies and the 6 x d/16 tcgen05 MMAs (small products
+// first); warps 0-3 read the fp32 accumulator from tensor memory, scale it and store their rows.
+// The accumulator is double-buffered, so the epilogue of one tile overlaps the copies and MMAs
+// of the next; shared memory holds one tile's operands (192 KB), reloaded as soon as the MMAs
+// that read them have completed.
 namespace sc {
-constexpr int kThreads = 128;
+constexpr int kThreads = 160;
 constexpr uint32_t kHalfBytes = 128 * 64 * 2;
 }
 
 template <int D>
 __global__ void __launch_bounds__(sc::kThreads, 1)
 score_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                float* __restrict__ scores, int nb, int BH, int score_stride, float sm_scale, void* workspace) {
+                float* __restrict__ scores, int nb, int BH, int score_stride, float sm_scale, int tiles_per_side,
+                void* workspace) {
     using namespace sc;
     constexpr uint32_t kPartBytes = 128 * D * 2;                  // one 128 x d operand tile
     constexpr int kHalves = D / 64;
     extern __shared__ __align__(1024) unsigned char sc_smem[];
     unsigned char* a_parts = sc_smem;                              // [3][kPartBytes]
     unsigned char* b_parts = sc_smem + 3 * kPartBytes;             // [3][kPartBytes]
-    __shared__ unsigned long long bar_full, bar_done;
+    __shared__ unsigned long long bar_full, bar_mma[2], bar_free[2];
     __shared__ uint32_t tmem_slot;
     __shared__ int abort_flag;
 
-    const int tid = threadIdx.x, warp = tid >> 5;
-    const int j0 = blockIdx.x * 128, i0 = blockIdx.y * 128, bh = blockIdx.z;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int per_head = tiles_per_side * tiles_per_side;
+    const int n_tiles = per_head * BH;
     if ((smem_u32(sc_smem) & 1023u) != 0u) {
         if (tid == 0) report_error(workspace, FVATTN_ERR_CUDA, 0x1025u);
         return;
     }
     if (tid == 0) {
         mbar_init(smem_u32(&bar_full), 1);
-        mbar_init(smem_u32(&bar_done), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&bar_mma[i]), 1); mbar_init(smem_u32(&bar_free[i]), 4); }
         abort_flag = 0;
         fence_barrier_init();
     }
     if (warp == 0) {
-        tmem_alloc(smem_u32(&tmem_slot), 128);
+        tmem_alloc(smem_u32(&tmem_slot), 256);
         tmem_relinquish();
     }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_slot;
+    bool failed = false;
 
-    bool ok = true;
-    if (tid == 0) {
-        const uint32_t bar = smem_u32(&bar_full);
-        mbar_expect_tx(bar, 6 * kPartBytes);
-        for (int part = 0; part < 3; ++part)
-            for (int h = 0; h < kHalves; ++h) {
-                tma_load_3d(smem_u32(a_parts) + part * kPartBytes + h * kHalfBytes, &map_q, 64 * h, i0, part * BH + bh, bar);
-                tma_load_3d(smem_u32(b_parts) + part * kPartBytes + h * kHalfBytes, &map_k, 64 * h, j0, part * BH + bh, bar);
-            }
-        ok = mbar_wait(bar, 0, &abort_flag);
-        if (ok) {
-            tc_fence_after();
+    if (warp == 4) {
+        if (lane == 0) {
+            // ---- copies + MMAs ------------------------------------------------------------------
             constexpr uint32_t idesc = make_idesc_bf16(128, 128, false);
-            // (query part, key part), smallest products first
-            const int combo[6][2] = {{0, 2}, {1, 1}, {2, 0}, {0, 1}, {1, 0}, {0, 0}};
-            bool first = true;
+            const int combo[6][2] = {{0, 2}, {1, 1}, {2, 0}, {0, 1}, {1, 0}, {0, 0}};   // (query part, key part)
+            uint32_t k = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++k) {
+                const int bh = tile / per_head, rem = tile - bh * per_head;
+                const int i0 = (rem / tiles_per_side) * 128, j0 = (rem % tiles_per_side) * 128;
+                const uint32_t acc = k & 1u;
+                // the operands of the previous tile are free once its MMAs have completed
+                if (k >= 1) ok = mbar_wait(smem_u32(&bar_mma[acc ^ 1u]), ((k - 1u) >> 1) & 1u, &abort_flag);
+                if (!ok) break;
+                const uint32_t bar = smem_u32(&bar_full);
+                mbar_expect_tx(bar, 6 * kPartBytes);
+                for (int part = 0; part < 3; ++part)
+                    for (int h = 0; h < kHalves; ++h) {
+                        tma_load_3d(smem_u32(a_parts) + part * kPartBytes + h * kHalfBytes, &map_q, 64 * h, i0, part * BH + bh, bar);
+                        tma_load_3d(smem_u32(b_parts) + part * kPartBytes + h * kHalfBytes, &map_k, 64 * h, j0, part * BH + bh, bar);
+                    }
+                ok = mbar_wait(bar, k & 1u, &abort_flag);
+                // the accumulator used two tiles ago must have been read out
+                if (ok && k >= 2) ok = mbar_wait(smem_u32(&bar_free[acc]), ((k - 2u) >> 1) & 1u, &abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                bool first = true;
 #pragma unroll
-            for (int cidx = 0; cidx < 6; ++cidx) {
-                const uint32_t sa = smem_u32(a_parts) + combo[cidx][0] * kPartBytes;
-                const uint32_t sb = smem_u32(b_parts) + combo[cidx][1] * kPartBytes;
+                for (int cidx = 0; cidx < 6; ++cidx) {
+                    const uint32_t sa = smem_u32(a_parts) + combo[cidx][0] * kPartBytes;
+                    const uint32_t sb = smem_u32(b_parts) + combo[cidx][1] * kPartBytes;
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
-                    umma_ss(tmem, make_smem_desc_sw128(sa + off, 16, 1024), make_smem_desc_sw128(sb + off, 16, 1024),
-                            idesc, first ? 0u : 1u);
-                    first = false;
+                    for (int ks = 0; ks < D / 16; ++ks) {
+                        const uint32_t off = (uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u;
+                        umma_ss(tmem + 128u * acc, make_smem_desc_sw128(sa + off, 16, 1024),
+                                make_smem_desc_sw128(sb + off, 16, 1024), idesc, first ? 0u : 1u);
+                        first = false;
+                    }
                 }
+                umma_commit(smem_u32(&bar_mma[acc]));
             }
-            umma_commit(smem_u32(&bar_done));
-        } else {
-            abort_flag = 1;
+            failed = !ok;
         }
-    }
-    ok = mbar_wait(smem_u32(&bar_done), 0, &abort_flag);
-    if (__syncthreads_and(ok ? 1 : 0)) {
-        tc_fence_after();
-        const int i = i0 + tid;                                    // this thread's row = its TMEM lane
-        float* out = scores + ((int64_t)bh * nb + i) * score_stride + j0;
+    } else {
+        // ---- epilogue warps: row `tid` of every tile -------------------------------------------------
+        uint32_t k = 0;
+        bool ok = true;
         const uint32_t lane_addr = tmem + ((uint32_t)(warp * 32) << 16);
+        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++k) {
+            const int bh = tile / per_head, rem = tile - bh * per_head;
+            const int i0 = (rem / tiles_per_side) * 128, j0 = (rem % tiles_per_side) * 128;
+            const uint32_t acc = k & 1u;
+            ok = mbar_wait(smem_u32(&bar_mma[acc]), (k >> 1) & 1u, &abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const int i = i0 + tid;
+            float* out = scores + ((int64_t)bh * nb + i) * score_stride + j0;
 #pragma unroll
-        for (int ch = 0; ch < 4; ++ch) {
-            uint32_t r[32];
-            tmem_ld32(lane_addr + ch * 32, r);
-            tmem_wait_ld();
-            if (i < nb) {
+            for (int ch = 0; ch < 4; ++ch) {
+                uint32_t r[32];
+                tmem_ld32(lane_addr + 128u * acc + ch * 32, r);
+                tmem_wait_ld();
+                if (i < nb) {
 #pragma unroll
-                for (int c4 = 0; c4 < 32; c4 += 4) {
-                    if (j0 + ch * 32 + c4 < score_stride)           // score_stride is a multiple of 4
-                        *reinterpret_cast<float4*>(out + ch * 32 + c4) =
-                            make_float4(sm_scale * __uint_as_float(r[c4]), sm_scale * __uint_as_float(r[c4 + 1]),
-                                        sm_scale * __uint_as_float(r[c4 + 2]), sm_scale * __uint_as_float(r[c4 + 3]));
+                    for (int c4 = 0; c4 < 32; c4 += 4) {
+                        if (j0 + ch * 32 + c4 < score_stride)           // score_stride is a multiple of 4
+                            *reinterpret_cast<float4*>(out + ch * 32 + c4) =
+                                make_float4(sm_scale * __uint_as_float(r[c4]), sm_scale * __uint_as_float(r[c4 + 1]),
+                                            sm_scale * __uint_as_float(r[c4 + 2]), sm_scale * __uint_as_float(r[c4 + 3]));
+                    }
                 }
             }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bar_free[acc]));
         }
-    } else if (tid == 0) {
+        failed = !ok;
+    }
+    if (failed) {
+        abort_flag = 1;
         report_error(workspace, FVATTN_ERR_DEVICE_TIMEOUT, 0x9002u);
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
         tc_fence_after();
-        tmem_dealloc(tmem, 128);
+        tmem_dealloc(tmem, 256);
     }
 }
 
@@ -740,9 +771,11 @@ static fvattn_status_t launch_stages(const void* q_r, const void* k_r, int64_t B
     if (!make_split_map(&mq, qsplit, D, m.nb, BH) || !make_split_map(&mk, ksplit, D, m.nb, BH)) return FVATTN_ERR_CUDA;
     const size_t smem = 6 * (size_t)128 * D * 2;
     FVATTN_CUDA_OK(cudaFuncSetAttribute(score_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-    const unsigned tiles = (unsigned)((m.nb + 127) / 128);
-    score_tc_kernel<D><<<dim3(tiles, tiles, (unsigned)BH), sc::kThreads, smem, s>>>(mq, mk, scores, m.nb, (int)BH,
-                                                                                  score_stride, sm_scale, workspace);
+    const int tiles = (m.nb + 127) / 128;
+    const int64_t n_tiles = (int64_t)tiles * tiles * BH;
+    const unsigned grid = (unsigned)(n_tiles < sms ? n_tiles : sms);
+    score_tc_kernel<D><<<grid, sc::kThreads, smem, s>>>(mq, mk, scores, m.nb, (int)BH, score_stride, sm_scale, tiles,
+                                                       workspace);
     return launch_status();
 }
 
