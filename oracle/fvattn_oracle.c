@@ -28,8 +28,9 @@
  *   before the floor; floor = integer block count clamped to nb; padded tokens
  *   are zero rows, left out of pooling, masked as keys, zero as queries.
  *
- * Parity pins: every function here is pinned by tests/test_oracle_pins.py
- * (closed forms, invariants, brute force, library routines).  The paper prints
+ * Parity pins: every function here (routing, attention, reorder, pooling, the
+ * augmentation step and the Hilbert walk further down) is pinned by
+ * tests/test_oracle_pins.py (closed forms, invariants, brute force, library routines).  The paper prints
  * no worked numeric example for this path, so numeric parity with the paper's
  * own implementation is unpinned; only the definitions are pinned.
  *

@@ -67,7 +67,7 @@ __host__ __device__ inline int block_valid_tokens(const GridDims& m, int blk) {
 
 // ---- workspace ------------------------------------------------------------------------
 // [0, 256): header.  word 0 = sticky status, word 1 = detail, word 2 = tile counter of the
-// persistent attention kernel, word 3 = CTAs that finished (used to re-arm the counter).
+// persistent attention kernel (re-armed by the tile-order kernel that precedes every launch).
 constexpr size_t kWsHeaderBytes = 256;
 constexpr int kMaxBlocks = 4096;
 
