@@ -341,9 +341,9 @@ void oracle_augment(const uint16_t* order, int32_t* counts, const int32_t* extra
  * tiles == NULL: all (bh, i) tiles, out is [BH, N_pad, d].
  * tiles != NULL: tiles[t] = bh * nb + i, out is [n_tiles, Bs, d].
  */
-void oracle_sparse_attn(const uint16_t* q_r, const uint16_t* k_r, const uint16_t* v_r, const uint16_t* idx,
-                        const int32_t* counts, int32_t BH, int32_t d, const ogrid_t* g, double sm_scale,
-                        const int64_t* tiles, int64_t n_tiles, double* out) {
+static void sparse_attn_impl(const uint16_t* q_r, const uint16_t* k_r, const uint16_t* v_r, const double* v_f64,
+                             const uint16_t* idx, const int32_t* counts, int32_t BH, int32_t d, const ogrid_t* g,
+                             double sm_scale, const int64_t* tiles, int64_t n_tiles, double* out) {
     int32_t nb = oracle_num_blocks(g), bs = oracle_block_tokens(g);
     int64_t n_pad = oracle_padded_tokens(g);
     uint8_t* valid = (uint8_t*)malloc((size_t)n_pad);
@@ -399,8 +399,9 @@ void oracle_sparse_attn(const uint16_t* q_r, const uint16_t* k_r, const uint16_t
                         int64_t rk = base + oo;
                         if (!valid[rk]) continue;
                         double w = z[rk] / denom;
-                        const uint16_t* vrow = v_r + ((int64_t)bh * n_pad + rk) * d;
-                        for (int32_t cc = 0; cc < d; ++cc) orow[cc] += w * bf16_to_f64(vrow[cc]);
+                        int64_t vbase = ((int64_t)bh * n_pad + rk) * d;
+                        for (int32_t cc = 0; cc < d; ++cc)
+                            orow[cc] += w * (v_f64 ? v_f64[vbase + cc] : bf16_to_f64(v_r[vbase + cc]));
                     }
                 }
             }
@@ -409,6 +410,19 @@ void oracle_sparse_attn(const uint16_t* q_r, const uint16_t* k_r, const uint16_t
         free(qd);
     }
     free(valid);
+}
+
+void oracle_sparse_attn(const uint16_t* q_r, const uint16_t* k_r, const uint16_t* v_r, const uint16_t* idx,
+                        const int32_t* counts, int32_t BH, int32_t d, const ogrid_t* g, double sm_scale,
+                        const int64_t* tiles, int64_t n_tiles, double* out) {
+    sparse_attn_impl(q_r, k_r, v_r, NULL, idx, counts, BH, d, g, sm_scale, tiles, n_tiles, out);
+}
+
+/* Same definition with V given as real numbers (the dequantised values of a quantised V). */
+void oracle_sparse_attn_vf64(const uint16_t* q_r, const uint16_t* k_r, const double* v_f64, const uint16_t* idx,
+                             const int32_t* counts, int32_t BH, int32_t d, const ogrid_t* g, double sm_scale,
+                             const int64_t* tiles, int64_t n_tiles, double* out) {
+    sparse_attn_impl(q_r, k_r, NULL, v_f64, idx, counts, BH, d, g, sm_scale, tiles, n_tiles, out);
 }
 
 /*
@@ -456,4 +470,67 @@ void oracle_hilbert_row_tokens(int32_t T, int32_t Y, int32_t X, int32_t bs, int3
             row_token[r++] = (int32_t)(((int64_t)c[0] * Y + c[1]) * X + c[2]);
     }
     for (; r < n_rows; ++r) row_token[r] = -1;
+}
+
+/*
+ * Quantised V (Sec. 3.4 mentions a mandatory V quantisation in the paper's kernel; the format is
+ * not stated).  Reading: per (batch, head) symmetric scaling into FP8 E4M3 (4 exponent bits, bias 7,
+ * 3 mantissa bits, largest finite value 448, no infinities):
+ *   scale = max |V| over the head's valid and padding rows / 448      (1 if the head is all zero)
+ *   code  = E4M3 nearest-even of V / scale, saturating
+ * The decision of every code is taken in fp32, the precision the CUDA kernel uses, so that the
+ * codes can be compared bit for bit: scale and the quotient are single-precision operations.
+ * Dequantised value = decode(code) * scale.
+ */
+static float e4m3_decode(uint8_t c) {
+    int sign = c >> 7, e = (c >> 3) & 15, m = c & 7;
+    float v = e == 0 ? ldexpf((float)m, -9) : ldexpf((float)(8 + m), e - 10);   /* subnormals: m * 2^-9 */
+    return sign ? -v : v;
+}
+
+static uint8_t e4m3_encode(float x) {
+    uint8_t sign = signbit(x) ? 0x80 : 0;
+    float a = fabsf(x);
+    if (!(a == a)) return sign | 0x7f;          /* NaN */
+    if (a >= 448.0f) return sign | 0x7e;        /* saturate to the largest finite value */
+    /* nearest representable magnitude, ties to the even code: walk the 127 finite codes */
+    uint8_t best = 0;
+    float best_err = a;                          /* code 0 = 0.0 */
+    for (int c = 1; c <= 0x7e; ++c) {
+        float err = fabsf(e4m3_decode((uint8_t)c) - a);
+        if (err < best_err || (err == best_err && (c & 1) == 0)) {
+            best = (uint8_t)c;
+            best_err = err;
+        }
+    }
+    return sign | best;
+}
+
+void oracle_e4m3_encode(const float* x, int64_t n, uint8_t* codes) {
+    for (int64_t i = 0; i < n; ++i) codes[i] = e4m3_encode(x[i]);
+}
+
+void oracle_e4m3_decode(const uint8_t* codes, int64_t n, float* x) {
+    for (int64_t i = 0; i < n; ++i) x[i] = e4m3_decode(codes[i]);
+}
+
+/* v_r: [BH, n_pad, d] bf16 -> codes [BH, n_pad, d] u8, scale [BH] f32, dequantised values [BH, n_pad, d] f64 */
+void oracle_quantize_v(const uint16_t* v_r, int32_t BH, int64_t n_pad, int32_t d, uint8_t* codes, float* scale,
+                       double* dequant) {
+#pragma omp parallel for schedule(static)
+    for (int32_t bh = 0; bh < BH; ++bh) {
+        const uint16_t* v = v_r + (int64_t)bh * n_pad * d;
+        float amax = 0.0f;
+        for (int64_t i = 0; i < n_pad * d; ++i) {
+            float a = fabsf((float)bf16_to_f64(v[i]));
+            if (a > amax) amax = a;
+        }
+        float sc = amax > 0.0f ? amax / 448.0f : 1.0f;
+        scale[bh] = sc;
+        for (int64_t i = 0; i < n_pad * d; ++i) {
+            uint8_t c = e4m3_encode((float)bf16_to_f64(v[i]) / sc);
+            codes[(int64_t)bh * n_pad * d + i] = c;
+            if (dequant) dequant[(int64_t)bh * n_pad * d + i] = (double)e4m3_decode(c) * (double)sc;
+        }
+    }
 }

@@ -200,6 +200,54 @@ def augment(res: RouteResult, extra: np.ndarray) -> RouteResult:
                        order=res.order, cum_at=res.cum_at, cum_before=res.cum_before, gap=res.gap)
 
 
+def e4m3_encode(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint8)
+    lib().oracle_e4m3_encode(_p(x), ctypes.c_int64(x.size), _p(out))
+    return out
+
+
+def e4m3_decode(codes: np.ndarray) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.empty(codes.shape, dtype=np.float32)
+    lib().oracle_e4m3_decode(_p(codes), ctypes.c_int64(codes.size), _p(out))
+    return out
+
+
+def quantize_v(v_r: np.ndarray):
+    """v_r [BH, N_pad, d] uint16 (bf16 bits) -> (codes uint8, scale float32 [BH], dequantised float64)."""
+    v_r = _u16(v_r)
+    BH, n_pad, d = v_r.shape
+    codes = np.empty((BH, n_pad, d), dtype=np.uint8)
+    scale = np.empty((BH,), dtype=np.float32)
+    deq = np.empty((BH, n_pad, d), dtype=np.float64)
+    lib().oracle_quantize_v(_p(v_r), ctypes.c_int32(BH), ctypes.c_int64(n_pad), ctypes.c_int32(d), _p(codes),
+                            _p(scale), _p(deq))
+    return codes, scale, deq
+
+
+def sparse_attn_vf64(q_r, k_r, v_f64, idx, counts, g: Grid, sm_scale: float, tiles=None) -> np.ndarray:
+    """sparse_attn with V given as float64 values [BH, N_pad, d] (e.g. a dequantised V)."""
+    q_r, k_r = _u16(q_r), _u16(k_r)
+    BH, n_pad, d = q_r.shape
+    nb, bs = num_blocks(g), block_tokens(g)
+    v_f64 = np.ascontiguousarray(v_f64, dtype=np.float64)
+    assert v_f64.shape == q_r.shape
+    idx = np.ascontiguousarray(idx, dtype=np.uint16)
+    counts = np.ascontiguousarray(counts, dtype=np.int32)
+    if tiles is None:
+        out = np.empty((BH, n_pad, d), dtype=np.float64)
+        n_tiles = 0
+    else:
+        tiles = np.ascontiguousarray(tiles, dtype=np.int64)
+        n_tiles = tiles.shape[0]
+        out = np.empty((n_tiles, bs, d), dtype=np.float64)
+    lib().oracle_sparse_attn_vf64(_p(q_r), _p(k_r), _p(v_f64), _p(idx), _p(counts), ctypes.c_int32(BH),
+                                  ctypes.c_int32(d), ctypes.byref(g.c()), ctypes.c_double(sm_scale), _p(tiles),
+                                  ctypes.c_int64(n_tiles), _p(out))
+    return out
+
+
 def hilbert_row_tokens(T: int, Y: int, X: int, block_tokens: int) -> np.ndarray:
     """Token at every position of the 3-D Hilbert curve through the grid (-1 on the padding rows)."""
     n = T * Y * X

@@ -301,6 +301,38 @@ def test_hilbert_rows_on_a_ragged_grid(shape, bs):
     assert (step == 1).mean() > 0.9
 
 
+# ---------------------------------------------------------------- quantised V (E4M3)
+def test_e4m3_codes_match_the_library_conversion():
+    """torch's float8_e4m3fn conversion (round to nearest even) on values inside the finite range, every
+    code decoded back, and the saturation at 448."""
+    rng = np.random.default_rng(0)
+    x = np.concatenate([rng.standard_normal(20000) * 100, rng.standard_normal(20000), rng.standard_normal(5000) * 1e-2,
+                        np.array([0.0, -0.0, 448.0, -448.0, 447.9, 2.0 ** -9, 2.0 ** -10, 3 * 2.0 ** -10])]).astype(np.float32)
+    x = x[np.abs(x) <= 448]
+    want = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = O.e4m3_encode(x)
+    same_value = O.e4m3_decode(got) == O.e4m3_decode(want)        # +0 / -0 codes decode alike
+    assert same_value.all()
+    codes = np.arange(256, dtype=np.uint8)
+    codes = codes[(codes & 0x7f) != 0x7f]                          # the two NaN codes
+    ref = torch.from_numpy(codes).view(torch.float8_e4m3fn).to(torch.float32).numpy()
+    np.testing.assert_array_equal(O.e4m3_decode(codes), ref)
+    assert O.e4m3_encode(np.array([1e6, -1e6], np.float32)).tolist() == [0x7e, 0xfe]    # saturates, no NaN
+
+
+def test_quantize_v_scale_and_error_bound():
+    cfg, g, q_r, k_r, v_r = _routing_inputs("tiny")
+    codes, scale, deq = O.quantize_v(v_r)
+    vf = bits_to_f64(v_r)
+    np.testing.assert_allclose(scale, np.abs(vf).max(axis=(1, 2)).astype(np.float32) / np.float32(448.0), rtol=1e-7)
+    # E4M3 keeps 3 mantissa bits: relative error <= 2^-4 on normal values, absolute <= scale * 2^-10 below
+    err = np.abs(deq - vf)
+    bound = np.maximum(np.abs(vf) * 2.0 ** -4, scale[:, None, None].astype(np.float64) * 2.0 ** -10)
+    assert (err <= bound * (1 + 1e-6)).all()
+    # the largest magnitude of each head maps to +-448 exactly
+    assert (np.abs(O.e4m3_decode(codes)).max(axis=(1, 2)) == 448).all()
+
+
 # ---------------------------------------------------------------- augmentation (Sec. 3.3)
 def test_augmentation_appends_the_next_ranks_and_only_grows_the_mask():
     cfg, g, q_r, k_r, _ = _routing_inputs("small")
