@@ -333,6 +333,16 @@ def run_ours(args):
     }
     if not args.no_dense:
         extra.update(dense_baselines(fv, layer, cfg, g, q, k, v, attn_ms, torch))
+    if args.fp8v:
+        v8, vs = fv.quantize_v(layer.v_r, g, layer.workspace)
+        f8 = lambda: fv.sparse_attn_fp8v(layer.q_r, layer.k_r, v8, vs, layer.routing.idx, layer.routing.counts, g,
+                                         layer.sm_scale, layer.workspace, layer.o_r)
+        qv = lambda: fv.quantize_v(layer.v_r, g, layer.workspace)
+        f8()
+        t8 = time_steps(f8, 5, torch) / 5
+        extra.update({"fp8v_attn_ms": t8, "fp8v_attn_tflops": flops / (t8 * 1e-3) / 1e12,
+                      "fp8v_quantize_ms": time_steps(qv, 5, torch) / 5})
+        del v8, vs
     cpu = None
     if not args.no_cpu_baseline and world == 1 or (world > 1 and not args.no_cpu_baseline and args.cpu_baseline_multi):
         cpu = oracle_sample(synth.CONFIGS[args.workload], budget_s=12.0)
@@ -461,6 +471,7 @@ def main():
     ap.add_argument("--no-dense", action="store_true", help="skip the dense baselines")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline-multi", action="store_true", help="also time the oracle when N > 1")
+    ap.add_argument("--fp8v", action="store_true", help="also time the quantised-V attention variant")
     ap.add_argument("--sweep", action="store_true", help="run the 720p layer x p sweep instead of the timed step")
     ap.add_argument("--sweep-layers", type=int, default=40)
     ap.add_argument("--sweep-dense-layers", type=int, default=4)

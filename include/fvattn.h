@@ -167,6 +167,26 @@ fvattn_status_t fvattn_sparse_attn(const void* q_r, const void* k_r, const void*
                                    const fvattn_grid_t* grid, float sm_scale, void* o_r, void* workspace,
                                    size_t workspace_bytes, fvattn_stream_t stream);
 
+/*
+ * Quantised-V variant (Sec. 3.4: the paper's kernel quantises V before the block-sparse attention;
+ * the format is not stated - this is the reading built here).
+ *
+ * fvattn_quantize_v: V -> FP8 E4M3 codes with one scale per (batch, head):
+ *   scale[b,h] = max |V[b,h]| / 448 (1 if all zero), code = nearest-even E4M3 of V / scale, saturating,
+ *   every step in fp32.   v_r bf16 [B,H,N_pad,d] -> v8 u8 [B,H,N_pad,d], v_scale f32 [B,H].
+ * fvattn_sparse_attn_fp8v: fvattn_sparse_attn with V read as v8 * v_scale.  The softmax weights are
+ *   handed to the second MMA as E4M3 too (3 mantissa bits), so the result carries a relative error of
+ *   a few per cent per weight: tested to max-abs 0.2 / mean-abs 5e-3 against exact attention over the
+ *   dequantised V (observed 0.11 / 1.6e-3).  Bs = d = 128 only.  Same workspace as fvattn_sparse_attn.
+ */
+fvattn_status_t fvattn_quantize_v(const void* v_r, int32_t B, int32_t H, int32_t d, const fvattn_grid_t* grid,
+                                  void* v8, float* v_scale, void* workspace, size_t workspace_bytes,
+                                  fvattn_stream_t stream);
+fvattn_status_t fvattn_sparse_attn_fp8v(const void* q_r, const void* k_r, const void* v8, const float* v_scale,
+                                        const uint16_t* idx, const int32_t* counts, int32_t B, int32_t H, int32_t d,
+                                        const fvattn_grid_t* grid, float sm_scale, void* o_r, void* workspace,
+                                        size_t workspace_bytes, fvattn_stream_t stream);
+
 /* Same contract as fvattn_sparse_attn, computed by the plain CUDA-core kernel (no tensor
  * cores).  fvattn_sparse_attn uses it for shapes other than Bs = d = 128; exported so the
  * two kernels can be compared on a GPU. */

@@ -24,7 +24,7 @@ EXPORTS = (
     "fvattn_num_blocks", "fvattn_block_tokens", "fvattn_padded_tokens", "fvattn_workspace_bytes",
     "fvattn_workspace_init", "fvattn_reorder", "fvattn_inverse_reorder", "fvattn_route",
     "fvattn_hilbert_row_tokens", "fvattn_reorder_by_table", "fvattn_inverse_reorder_by_table",
-    "fvattn_augment", "fvattn_sparse_attn", "fvattn_sparse_attn_simt", "fvattn_sparse_attn_noalloc", "fvattn_tile_order",
+    "fvattn_quantize_v", "fvattn_sparse_attn_fp8v", "fvattn_augment", "fvattn_sparse_attn", "fvattn_sparse_attn_simt", "fvattn_sparse_attn_noalloc", "fvattn_tile_order",
     "fvattn_device_status",
     "fvattn_status_string",
 )
@@ -302,6 +302,32 @@ def sparse_attn_noalloc(q_r, k_r, v_r, idx, counts, grid: Grid, sm_scale: float 
     _check(lib().fvattn_sparse_attn_noalloc(_ptr(q_r), _ptr(k_r), _ptr(v_r), _ptr(idx), _ptr(counts), B, H, d,
                                             ctypes.byref(grid.c()), ctypes.c_float(sm_scale), _ptr(out),
                                             _ptr(status_out), _stream()), "fvattn_sparse_attn_noalloc")
+    return out
+
+
+def quantize_v(v_r: torch.Tensor, grid: Grid, workspace: torch.Tensor):
+    """V [B, H, N_pad, d] bf16 -> (E4M3 codes uint8 [B, H, N_pad, d], scale float32 [B, H])."""
+    _need_cuda(v_r, workspace)
+    B, H, n_pad, d = v_r.shape
+    v8 = torch.empty(B, H, n_pad, d, dtype=torch.uint8, device=v_r.device)
+    scale = torch.empty(B, H, dtype=torch.float32, device=v_r.device)
+    _check(lib().fvattn_quantize_v(_ptr(v_r), B, H, d, ctypes.byref(grid.c()), _ptr(v8), _ptr(scale), _ptr(workspace),
+                                   ctypes.c_size_t(workspace.numel()), _stream()), "fvattn_quantize_v")
+    return v8, scale
+
+
+def sparse_attn_fp8v(q_r, k_r, v8, v_scale, idx, counts, grid: Grid, sm_scale: float | None, workspace: torch.Tensor,
+                     out: torch.Tensor | None = None) -> torch.Tensor:
+    """Block-sparse attention with V as E4M3 codes and per-head scales (Bs = d = 128)."""
+    _need_cuda(q_r, k_r, v8, v_scale, idx, counts, workspace)
+    B, H, n_pad, d = q_r.shape
+    if sm_scale is None:
+        sm_scale = 1.0 / math.sqrt(d)
+    if out is None:
+        out = torch.empty_like(q_r)
+    _check(lib().fvattn_sparse_attn_fp8v(_ptr(q_r), _ptr(k_r), _ptr(v8), _ptr(v_scale), _ptr(idx), _ptr(counts), B, H, d,
+                                         ctypes.byref(grid.c()), ctypes.c_float(sm_scale), _ptr(out), _ptr(workspace),
+                                         ctypes.c_size_t(workspace.numel()), _stream()), "fvattn_sparse_attn_fp8v")
     return out
 
 

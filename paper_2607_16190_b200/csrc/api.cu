@@ -179,10 +179,43 @@ fvattn_status_t fvattn_sparse_attn(const void* q_r, const void* k_r, const void*
     st = launch_tile_order(counts, BH, m.nb, order, workspace, (cudaStream_t)stream);
     if (st != FVATTN_OK) return st;
     if (m.bs == 128 && d == 128)
-        return launch_attn_tc(q_r, k_r, v_r, idx, counts, BH, m, sm_scale, o_r, order, workspace,
+        return launch_attn_tc(q_r, k_r, v_r, idx, counts, BH, m, sm_scale, o_r, order, workspace, nullptr,
                               (cudaStream_t)stream);
     return launch_attn_simt(q_r, k_r, v_r, idx, counts, BH, d, m, sm_scale, o_r, order, workspace,
                             (cudaStream_t)stream);
+}
+
+fvattn_status_t fvattn_quantize_v(const void* v_r, int32_t B, int32_t H, int32_t d, const fvattn_grid_t* grid,
+                                  void* v8, float* v_scale, void* workspace, size_t workspace_bytes,
+                                  fvattn_stream_t stream) {
+    if (!v_r || !v8 || !v_scale || !workspace || !grid_ok(grid) || B <= 0 || H <= 0) return FVATTN_ERR_INVALID_ARG;
+    GridDims m = make_dims(*grid);
+    if (!shape_ok(d, m)) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    const int64_t BH = (int64_t)B * H;
+    if (BH > 65535) return FVATTN_ERR_UNSUPPORTED_SHAPE;
+    if (!aligned(v_r, 16) || !aligned(v8, 16) || !aligned(v_scale, 4) || !aligned(workspace, 256))
+        return FVATTN_ERR_INVALID_ARG;
+    if (workspace_bytes < attn_ws(BH, m.nb).total) return FVATTN_ERR_WORKSPACE_TOO_SMALL;
+    unsigned int* amax = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) + attn_ws(BH, m.nb).head_sum);
+    return launch_quantize_v(v_r, BH, m.n_pad * d, v8, v_scale, amax, (cudaStream_t)stream);
+}
+
+fvattn_status_t fvattn_sparse_attn_fp8v(const void* q_r, const void* k_r, const void* v8, const float* v_scale,
+                                        const uint16_t* idx, const int32_t* counts, int32_t B, int32_t H, int32_t d,
+                                        const fvattn_grid_t* grid, float sm_scale, void* o_r, void* workspace,
+                                        size_t workspace_bytes, fvattn_stream_t stream) {
+    fvattn_status_t st = check_attn_args(q_r, k_r, v8, idx, counts, B, H, d, grid, sm_scale, o_r, workspace,
+                                         workspace_bytes);
+    if (st != FVATTN_OK) return st;
+    if (!v_scale || !aligned(v_scale, 4)) return FVATTN_ERR_INVALID_ARG;
+    GridDims m = make_dims(*grid);
+    if (m.bs != 128 || d != 128) return FVATTN_ERR_UNSUPPORTED_SHAPE;   // tensor-core kernel only
+    const int64_t BH = (int64_t)B * H;
+    uint32_t* order = reinterpret_cast<uint32_t*>(static_cast<char*>(workspace) + attn_ws(BH, m.nb).order);
+    st = launch_tile_order(counts, BH, m.nb, order, workspace, (cudaStream_t)stream);
+    if (st != FVATTN_OK) return st;
+    return launch_attn_tc(q_r, k_r, v8, idx, counts, BH, m, sm_scale, o_r, order, workspace, v_scale,
+                          (cudaStream_t)stream);
 }
 
 fvattn_status_t fvattn_device_status(const void* workspace, fvattn_stream_t stream) {

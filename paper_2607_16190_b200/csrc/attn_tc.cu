@@ -25,6 +25,8 @@
 // Every wait is a bounded mbarrier wait; when one runs out the CTA records
 // FVATTN_ERR_DEVICE_TIMEOUT in the workspace, every role leaves its loop, tensor memory is
 // freed and the kernel returns.
+#include <cuda_fp8.h>
+
 #include "common.cuh"
 #include "sm100_ptx.cuh"
 
@@ -105,12 +107,16 @@ key_mask_kernel(GridDims m, uint32_t* __restrict__ kmask) {
     if ((threadIdx.x & 31) == 0) kmask[blockIdx.x * 4 + (threadIdx.x >> 5)] = bal;
 }
 
+// kV8: V is FP8 E4M3 with one scale per (batch, head) (written by fvattn_quantize_v); P is then handed
+// to the second MMA as E4M3 too (kind::f8f6f4, K = 32 per instruction), and the output is multiplied by
+// the head's scale.  Everything else is identical to the bf16 path.
+template <bool kV8>
 __global__ void __launch_bounds__(tc::kThreads, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                const __grid_constant__ CUtensorMap map_v, const uint16_t* __restrict__ idx,
                const int32_t* __restrict__ counts, GridDims m, float sm_scale, __nv_bfloat16* __restrict__ o_r,
                const uint32_t* __restrict__ order, const uint4* __restrict__ kmask, int has_pad, int n_tiles,
-               void* workspace) {
+               void* workspace, const float* __restrict__ v_scale) {
     using namespace tc;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     Smem& sm = *reinterpret_cast<Smem*>(smem_raw);
@@ -260,9 +266,14 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                             ok = mbar_wait(smem_u32(&sm.v_empty[vs]), ((vn / VS) & 1u) ^ 1u, abort_flag);
                             if (ok) {
                                 const uint32_t bar = smem_u32(&sm.v_full[vs]);
-                                mbar_expect_tx(bar, kTileBytes);
-                                tma_load_2d(smem_u32(sm.v[vs]), &map_v, 0, krow, bar);
-                                tma_load_2d(smem_u32(sm.v[vs]) + kHalfBytes, &map_v, 64, krow, bar);
+                                if constexpr (kV8) {      // 128 keys x 128 one-byte columns: a single 16 KB box
+                                    mbar_expect_tx(bar, kHalfBytes);
+                                    tma_load_2d(smem_u32(sm.v[vs]), &map_v, 0, krow, bar);
+                                } else {
+                                    mbar_expect_tx(bar, kTileBytes);
+                                    tma_load_2d(smem_u32(sm.v[vs]), &map_v, 0, krow, bar);
+                                    tma_load_2d(smem_u32(sm.v[vs]) + kHalfBytes, &map_v, 64, krow, bar);
+                                }
                             }
                         }
                         ++vn;
@@ -336,10 +347,20 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         tc_fence_after();
                         const uint32_t vlo = v_lo0 + st * (kTileBytes >> 4);
                         const uint32_t tOb = tmem + kColO + 128u * b, tPb = tmem + kColS + 128u * b;
+                        if constexpr (kV8) {
+                            // 4 steps of 32 keys: P is 4 E4M3 per tensor-memory column, V rows are 128 B apart
+                            constexpr uint32_t idesc_pv8 = make_idesc_e4m3(128, 128);
+                            const uint32_t vlo8 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.v[st]), 16, 1024);
 #pragma unroll
-                        for (int ks = 0; ks < BS / 16; ++ks)
-                            umma_ts(tOb, tPb + ks * 8, ((uint64_t)desc_hi << 32) | (vlo + (uint32_t)ks * (2048u >> 4)), idesc_pv,
-                                    (t >= 2 || ks > 0) ? 1u : 0u);
+                            for (int ks = 0; ks < BS / 32; ++ks)
+                                umma_ts_f8(tOb, tPb + ks * 8, ((uint64_t)desc_hi << 32) | (vlo8 + (uint32_t)ks * (4096u >> 4)),
+                                           idesc_pv8, (t >= 2 || ks > 0) ? 1u : 0u);
+                        } else {
+#pragma unroll
+                            for (int ks = 0; ks < BS / 16; ++ks)
+                                umma_ts(tOb, tPb + ks * 8, ((uint64_t)desc_hi << 32) | (vlo + (uint32_t)ks * (2048u >> 4)),
+                                        idesc_pv, (t >= 2 || ks > 0) ? 1u : 0u);
+                        }
                         umma_commit(smem_u32(&sm.v_empty[st]));
                         umma_commit(smem_u32(&sm.pv_done[b]));
                         ++cnt;
@@ -440,26 +461,44 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 }
                 const float moff = (m_run == -INFINITY) ? 0.f : m_run * sl2;   // -inf only if no valid key yet
                 float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
-                uint32_t pk[64];
+                if constexpr (kV8) {
+                    uint32_t pk8[32];                              // 4 E4M3 weights per column, lowest key in the lowest byte
 #pragma unroll
-                for (int j = 0; j < 128; j += 4) {
-                    float e0 = __uint_as_float(s[j]), e1 = __uint_as_float(s[j + 1]), e2 = __uint_as_float(s[j + 2]),
-                          e3 = __uint_as_float(s[j + 3]);
-                    fma2(e0, e1, sl2, -moff);
-                    fma2(e2, e3, sl2, -moff);
-                    __nv_bfloat162 lo = __floats2bfloat162_rn(ex2(e0), ex2(e1));   // .x (low half) = even column
-                    __nv_bfloat162 hi = __floats2bfloat162_rn(ex2(e2), ex2(e3));
-                    const uint32_t wlo = *reinterpret_cast<uint32_t*>(&lo), whi = *reinterpret_cast<uint32_t*>(&hi);
-                    pk[j >> 1] = wlo;
-                    pk[(j >> 1) + 1] = whi;
-                    // the row sum takes the bf16-rounded weights the second MMA sees, so numerator and
-                    // denominator stay consistent (an exact weighted average of V)
-                    add_bf16_pair(sum0, sum1, wlo);
-                    add_bf16_pair(sum2, sum3, whi);
+                    for (int j = 0; j < 128; j += 4) {
+                        float e0 = __uint_as_float(s[j]), e1 = __uint_as_float(s[j + 1]), e2 = __uint_as_float(s[j + 2]),
+                              e3 = __uint_as_float(s[j + 3]);
+                        fma2(e0, e1, sl2, -moff);
+                        fma2(e2, e3, sl2, -moff);
+                        const float p0 = ex2(e0), p1 = ex2(e1), p2 = ex2(e2), p3 = ex2(e3);
+                        const uint32_t lo = __nv_cvt_float2_to_fp8x2(make_float2(p0, p1), __NV_SATFINITE, __NV_E4M3);
+                        const uint32_t hi = __nv_cvt_float2_to_fp8x2(make_float2(p2, p3), __NV_SATFINITE, __NV_E4M3);
+                        pk8[j >> 2] = lo | (hi << 16);
+                        sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
+                    }
+                    l_run += (sum0 + sum1) + (sum2 + sum3);
+                    tmem_st32(tS, pk8);
+                } else {
+                    uint32_t pk[64];
+#pragma unroll
+                    for (int j = 0; j < 128; j += 4) {
+                        float e0 = __uint_as_float(s[j]), e1 = __uint_as_float(s[j + 1]), e2 = __uint_as_float(s[j + 2]),
+                              e3 = __uint_as_float(s[j + 3]);
+                        fma2(e0, e1, sl2, -moff);
+                        fma2(e2, e3, sl2, -moff);
+                        __nv_bfloat162 lo = __floats2bfloat162_rn(ex2(e0), ex2(e1));   // .x (low half) = even column
+                        __nv_bfloat162 hi = __floats2bfloat162_rn(ex2(e2), ex2(e3));
+                        const uint32_t wlo = *reinterpret_cast<uint32_t*>(&lo), whi = *reinterpret_cast<uint32_t*>(&hi);
+                        pk[j >> 1] = wlo;
+                        pk[(j >> 1) + 1] = whi;
+                        // the row sum takes the bf16-rounded weights the second MMA sees, so numerator and
+                        // denominator stay consistent (an exact weighted average of V)
+                        add_bf16_pair(sum0, sum1, wlo);
+                        add_bf16_pair(sum2, sum3, whi);
+                    }
+                    l_run += (sum0 + sum1) + (sum2 + sum3);
+                    tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
+                    tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
                 }
-                l_run += (sum0 + sum1) + (sum2 + sum3);
-                tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-                tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -488,7 +527,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             int64_t token;
             const bool qvalid = !has_pad || row_to_token(m, i, row, &token);
             const float inv = (qvalid && lsum > 0.f) ? 1.f / lsum : 0.f;
-            const float f0 = w0 * inv, f1 = w1 * inv;
+            const float vs_h = kV8 ? v_scale[bh] : 1.f;
+            const float f0 = w0 * inv * vs_h, f1 = w1 * inv * vs_h;
             const uint32_t tO0 = tmem + lane_base + kColO + 64u * a;
             const uint32_t tO1 = tO0 + 128u;
 #pragma unroll
@@ -568,14 +608,29 @@ static bool make_tile_map(CUtensorMap* map, const void* base, uint64_t rows) {
     return r == CUDA_SUCCESS;
 }
 
+// [rows, 128] one-byte (E4M3) row-major tensor, box = 128 rows x 128 columns (128 B), 128-byte swizzle.
+static bool make_tile_map_u8(CUtensorMap* map, const void* base, uint64_t rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    cuuint64_t dims[2] = {(cuuint64_t)tc::D, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)tc::D};
+    cuuint32_t box[2] = {128, 128};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+// v_scale == NULL: v_r is bf16.  Otherwise v_r holds E4M3 codes and v_scale one fp32 scale per (batch, head).
 fvattn_status_t launch_attn_tc(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
                                const int32_t* counts, int64_t BH, const GridDims& m, float sm_scale, void* o_r,
-                               const uint32_t* order, void* workspace, cudaStream_t s) {
+                               const uint32_t* order, void* workspace, const float* v_scale, cudaStream_t s) {
     const uint64_t rows = (uint64_t)BH * (uint64_t)m.n_pad;
     if (rows > 0x7fffffffull) return FVATTN_ERR_UNSUPPORTED_SHAPE;   // TMA coordinates are 32-bit
     CUtensorMap mq, mk, mv;
-    if (!make_tile_map(&mq, q_r, rows) || !make_tile_map(&mk, k_r, rows) || !make_tile_map(&mv, v_r, rows))
-        return FVATTN_ERR_CUDA;
+    if (!make_tile_map(&mq, q_r, rows) || !make_tile_map(&mk, k_r, rows)) return FVATTN_ERR_CUDA;
+    if (!(v_scale ? make_tile_map_u8(&mv, v_r, rows) : make_tile_map(&mv, v_r, rows))) return FVATTN_ERR_CUDA;
     int dev = 0, sms = 0;
     FVATTN_CUDA_OK(cudaGetDevice(&dev));
     FVATTN_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
@@ -586,11 +641,19 @@ fvattn_status_t launch_attn_tc(const void* q_r, const void* k_r, const void* v_r
         if (launch_status() != FVATTN_OK) return FVATTN_ERR_CUDA;
     }
     const size_t smem = sizeof(tc::Smem);
-    FVATTN_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     const int n_tiles = (int)(BH * m.nb);
     const int grid = n_tiles < sms ? n_tiles : sms;
-    attn_tc_kernel<<<grid, tc::kThreads, smem, s>>>(mq, mk, mv, idx, counts, m, sm_scale, (__nv_bfloat16*)o_r, order,
-                                                   reinterpret_cast<const uint4*>(kmask), has_pad, n_tiles, workspace);
+    if (v_scale) {
+        FVATTN_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attn_tc_kernel<true><<<grid, tc::kThreads, smem, s>>>(mq, mk, mv, idx, counts, m, sm_scale, (__nv_bfloat16*)o_r,
+                                                             order, reinterpret_cast<const uint4*>(kmask), has_pad,
+                                                             n_tiles, workspace, v_scale);
+    } else {
+        FVATTN_CUDA_OK(cudaFuncSetAttribute(attn_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attn_tc_kernel<false><<<grid, tc::kThreads, smem, s>>>(mq, mk, mv, idx, counts, m, sm_scale, (__nv_bfloat16*)o_r,
+                                                              order, reinterpret_cast<const uint4*>(kmask), has_pad,
+                                                              n_tiles, workspace, nullptr);
+    }
     return launch_status();
 }
 

@@ -141,6 +141,8 @@ fvattn_status_t launch_route(const void* q_r, const void* k_r, int64_t BH, int d
                              float* head_load, void* workspace, cudaStream_t s);
 fvattn_status_t launch_augment(int64_t BH, int d, const GridDims& m, const int32_t* extra, uint32_t* mask_bits,
                                int32_t* counts, uint16_t* idx, float* head_load, void* workspace, cudaStream_t s);
+fvattn_status_t launch_quantize_v(const void* v_r, int64_t BH, int64_t elems_per_head, void* v8, float* v_scale,
+                                  unsigned int* amax_bits, cudaStream_t s);
 fvattn_status_t launch_tile_order(const int32_t* counts, int64_t BH, int nb, uint32_t* order, void* workspace,
                                   cudaStream_t s);
 fvattn_status_t launch_attn_simt(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
@@ -148,6 +150,6 @@ fvattn_status_t launch_attn_simt(const void* q_r, const void* k_r, const void* v
                                  void* o_r, const uint32_t* order, void* workspace, cudaStream_t s);
 fvattn_status_t launch_attn_tc(const void* q_r, const void* k_r, const void* v_r, const uint16_t* idx,
                                const int32_t* counts, int64_t BH, const GridDims& m, float sm_scale, void* o_r,
-                               const uint32_t* order, void* workspace, cudaStream_t s);
+                               const uint32_t* order, void* workspace, const float* v_scale, cudaStream_t s);
 
 } // namespace fvattn

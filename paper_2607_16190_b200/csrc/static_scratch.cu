@@ -69,7 +69,7 @@ extern "C" fvattn_status_t fvattn_sparse_attn_noalloc(const void* q_r, const voi
     st = launch_tile_order(counts, BH, m.nb, order, scratch, s);
     if (st != FVATTN_OK) return st;
     if (m.bs == 128 && d == 128)
-        st = launch_attn_tc(q_r, k_r, v_r, idx, counts, BH, m, sm_scale, o_r, order, scratch, s);
+        st = launch_attn_tc(q_r, k_r, v_r, idx, counts, BH, m, sm_scale, o_r, order, scratch, nullptr, s);
     else
         st = launch_attn_simt(q_r, k_r, v_r, idx, counts, BH, d, m, sm_scale, o_r, order, scratch, s);
     if (st != FVATTN_OK) return st;
