@@ -9,14 +9,17 @@
 //                 tcgen05 MMAs with the accumulators in tensor memory
 //   warps 4-7     softmax of the even retained blocks  (stream 0)
 //   warps 8-11    softmax of the odd retained blocks   (stream 1)
-// The retained blocks of a tile alternate between two independent streams, each with its own
-// S/P and O accumulators in tensor memory (4 x 128 columns = all 512) and its own running max
-// and sum, so the softmax of one stream overlaps the MMAs of the other; the two partial results
-// are merged once per tile (O = (O0 w0 + O1 w1) / (l0 w0 + l1 w1)).  One thread owns one query
-// row: it reads its S row from tensor memory, keeps a running max with lazy rescaling (O is only
-// rescaled when the max grows by more than 2^8), writes P back as bf16 over the S columns, and
-// the MMA thread feeds P from tensor memory as the A operand of the second MMA.  Padded keys of
-// edge blocks are masked to -inf from a per-block validity table; padded query rows give zero.
+// The retained blocks of a tile alternate between two independent streams, each with its own O
+// accumulator (128 columns) and two S/P slots of 64 columns in tensor memory (all 512 columns) and
+// its own running max and sum; the two partial results are merged once per tile
+// (O = (O0 w0 + O1 w1) / (l0 w0 + l1 w1)).  A block is pipelined as two half-blocks of 64 keys:
+// with two S slots per stream the QK MMA of a stream's next half-block is finished while its
+// softmax warps are still on the current one, and the online-softmax recurrence simply runs per
+// half-block.  One thread owns one query row: it reads 64 S values from tensor memory, keeps a
+// running max with lazy rescaling (O is only rescaled when the max grows by more than 2^8, after
+// the PV MMA in flight on it has completed), writes P back as bf16 over its S slot, and the PV
+// thread feeds P from tensor memory as the A operand of the second MMA.  Padded keys of edge
+// blocks are masked to -inf from a per-block validity table; padded query rows give zero.
 //
 // Shared-memory tiles use the 128-byte swizzle: a 128 x 128 bf16 tile is two TMA boxes of
 // 128 rows x 64 columns (16 KB each).  Q and K are K-major MMA operands; V (keys x d, d
@@ -44,7 +47,7 @@ constexpr int TS = 2;                               // tile-info ring depth
 constexpr uint32_t kHalfBytes = 128 * 64 * 2;       // one TMA box: 128 rows x 64 bf16
 constexpr uint32_t kTileBytes = 2 * kHalfBytes;     // 128 x 128 bf16
 constexpr uint32_t kTmemCols = 512;
-constexpr uint32_t kColS = 0;                       // S / P of stream a at kColS + 128 a
+constexpr uint32_t kColS = 0;                       // S / P of stream a, half-block slot h at kColS + 128 a + 64 h
 constexpr uint32_t kColO = 256;                     // O of stream a at kColO + 128 a
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kRescaleThreshold = 8.0f;           // log2 units
@@ -55,7 +58,7 @@ struct __align__(1024) Smem {
     unsigned char v[VS][kTileBytes];
     float ml[2][2][BS];                             // [stream][m, l][row]
     unsigned long long q_full, q_empty, k_full[KS], k_empty[KS], v_full[VS], v_empty[VS];
-    unsigned long long s_full[2], p_full[2], pv_done[2], o_full, o_free, ml_ready, ml_done, tile_full[TS], tile_empty[TS];
+    unsigned long long s_full[2][2], p_full[2][2], pv_done[2][2], o_full, o_free, ml_ready, ml_done, tile_full[TS], tile_empty[TS];
     int tile_id[TS];
     int tile_cnt[TS];
     uint32_t tmem_base;
@@ -135,11 +138,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
         mbar_init(smem_u32(&sm.q_empty), 1);
         for (int s = 0; s < KS; ++s) { mbar_init(smem_u32(&sm.k_full[s]), 1); mbar_init(smem_u32(&sm.k_empty[s]), 1); }
         for (int s = 0; s < VS; ++s) { mbar_init(smem_u32(&sm.v_full[s]), 1); mbar_init(smem_u32(&sm.v_empty[s]), 1); }
-        for (int a = 0; a < 2; ++a) {
-            mbar_init(smem_u32(&sm.s_full[a]), 1);
-            mbar_init(smem_u32(&sm.p_full[a]), 4);
-            mbar_init(smem_u32(&sm.pv_done[a]), 1);
-        }
+        for (int a = 0; a < 2; ++a)
+            for (int h = 0; h < 2; ++h) {
+                mbar_init(smem_u32(&sm.s_full[a][h]), 1);
+                mbar_init(smem_u32(&sm.p_full[a][h]), 4);
+                mbar_init(smem_u32(&sm.pv_done[a][h]), 1);
+            }
         mbar_init(smem_u32(&sm.o_full), 1);
         mbar_init(smem_u32(&sm.o_free), 8);
         mbar_init(smem_u32(&sm.ml_ready), 8);
@@ -286,8 +290,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             // ======================= MMA issuers: one thread for S = Q K^T, one for O += P V =============
             // Two threads on two schedulers halve the serial time per block that a single issuer spends on
             // barrier polls, commits and MMA instructions.  The only ordering the two need between them is
-            // that QK(t + 2) must not overwrite the S/P columns of stream a before PV(t) has read P: the
-            // QK thread waits for the completion of PV(t) (pv_done, a commit by the PV thread).
+            // that a QK MMA must not overwrite an S/P slot before the PV MMA of the slot's previous
+            // occupant has read P: the QK thread waits for that PV's completion (pv_done, a commit by the
+            // PV thread).
             constexpr uint32_t idesc_qk = make_idesc_bf16(128, 128, false);
             constexpr uint32_t idesc_pv = make_idesc_bf16(128, 128, true);
             // descriptor words that never change: high word (stride 1024 B, version, 128-byte swizzle);
@@ -296,6 +301,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const uint32_t q_lo = (uint32_t)make_smem_desc_sw128(smem_u32(sm.q), 16, 1024);
             const uint32_t k_lo0 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.k[0]), 16, 1024);
             const uint32_t v_lo0 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.v[0]), kHalfBytes, 1024);
+            // A retained block (128 keys) is pipelined as two half-blocks of 64 keys, and each stream owns two
+            // S/P slots (one per half): the QK MMA of a stream's next half-block is finished while its softmax
+            // warps are still on the current one, so in steady state they do not wait for the tensor pipe.
+            constexpr uint32_t idesc_qk64 = make_idesc_bf16(128, 64, false);
             uint32_t n = 0, ring = 0, qn = 0, cnt0 = 0, cnt1 = 0;   // cnt: blocks of each stream so far
             bool ok = true;
             const bool is_qk = warp == 1;
@@ -316,22 +325,29 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         const int a = t & 1;
                         uint32_t& cnt = a ? cnt1 : cnt0;
                         const uint32_t st = ring % KS, ph = (ring / KS) & 1u;
-                        // the previous block of this stream (possibly of the previous tile) must have been read by its PV
-                        if (cnt > 0) ok = mbar_wait(smem_u32(&sm.pv_done[a]), (cnt - 1u) & 1u, abort_flag);
-                        ok = ok && mbar_wait(smem_u32(&sm.k_full[st]), ph, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
+                        ok = mbar_wait(smem_u32(&sm.k_full[st]), ph, abort_flag);
                         const uint32_t klo = k_lo0 + st * (kTileBytes >> 4);
-                        const uint32_t tSa = tmem + kColS + 128u * a;
 #pragma unroll
-                        for (int ks = 0; ks < D / 16; ++ks) {
-                            const uint32_t off16 = ((uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u) >> 4;
-                            umma_ss(tSa, ((uint64_t)desc_hi << 32) | (q_lo + off16), ((uint64_t)desc_hi << 32) | (klo + off16),
-                                    idesc_qk, ks > 0 ? 1u : 0u);
+                        for (int half = 0; half < 2; ++half) {
+                            // the slot's previous occupant (this stream's previous block, same half) must have been
+                            // read by its PV
+                            if (ok && cnt > 0) ok = mbar_wait(smem_u32(&sm.pv_done[a][half]), (cnt - 1u) & 1u, abort_flag);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint32_t tSa = tmem + kColS + 128u * a + 64u * half;
+                            const uint32_t kh = klo + (uint32_t)half * (8192u >> 4);        // key rows 64 half ..
+#pragma unroll
+                            for (int ks = 0; ks < D / 16; ++ks) {
+                                const uint32_t off16 = ((uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u) >> 4;
+                                umma_ss(tSa, ((uint64_t)desc_hi << 32) | (q_lo + off16), ((uint64_t)desc_hi << 32) | (kh + off16),
+                                        idesc_qk64, ks > 0 ? 1u : 0u);
+                            }
+                            if (half == 1) {
+                                umma_commit(smem_u32(&sm.k_empty[st]));
+                                if (t == c - 1) umma_commit(smem_u32(&sm.q_empty));
+                            }
+                            umma_commit(smem_u32(&sm.s_full[a][half]));
                         }
-                        umma_commit(smem_u32(&sm.k_empty[st]));
-                        if (t == c - 1) umma_commit(smem_u32(&sm.q_empty));
-                        umma_commit(smem_u32(&sm.s_full[a]));
                         ++cnt;
                         ++ring;
                     }
@@ -340,29 +356,38 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         const int b = t & 1;
                         uint32_t& cnt = b ? cnt1 : cnt0;
                         const uint32_t st = ring % VS, ph = (ring / VS) & 1u;
-                        ok = mbar_wait(smem_u32(&sm.p_full[b]), cnt & 1u, abort_flag) &&
-                             mbar_wait(smem_u32(&sm.v_full[st]), ph, abort_flag);
-                        if (ok && t == 0) ok = mbar_wait(smem_u32(&sm.o_free), (qn & 1u) ^ 1u, abort_flag);
-                        if (!ok) break;
-                        tc_fence_after();
                         const uint32_t vlo = v_lo0 + st * (kTileBytes >> 4);
-                        const uint32_t tOb = tmem + kColO + 128u * b, tPb = tmem + kColS + 128u * b;
-                        if constexpr (kV8) {
-                            // 4 steps of 32 keys: P is 4 E4M3 per tensor-memory column, V rows are 128 B apart
-                            constexpr uint32_t idesc_pv8 = make_idesc_e4m3(128, 128);
-                            const uint32_t vlo8 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.v[st]), 16, 1024);
+                        const uint32_t vlo8 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.v[st]), 16, 1024);
+                        const uint32_t tOb = tmem + kColO + 128u * b;
 #pragma unroll
-                            for (int ks = 0; ks < BS / 32; ++ks)
-                                umma_ts_f8(tOb, tPb + ks * 8, ((uint64_t)desc_hi << 32) | (vlo8 + (uint32_t)ks * (4096u >> 4)),
-                                           idesc_pv8, (t >= 2 || ks > 0) ? 1u : 0u);
-                        } else {
+                        for (int half = 0; half < 2; ++half) {
+                            ok = ok && mbar_wait(smem_u32(&sm.p_full[b][half]), cnt & 1u, abort_flag);
+                            if (half == 0) {
+                                ok = ok && mbar_wait(smem_u32(&sm.v_full[st]), ph, abort_flag);
+                                if (ok && t == 0) ok = mbar_wait(smem_u32(&sm.o_free), (qn & 1u) ^ 1u, abort_flag);
+                            }
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint32_t tPb = tmem + kColS + 128u * b + 64u * half;
+                            const uint32_t first = (t < 2 && half == 0) ? 0u : 1u;       // overwrite O on a stream's first half-block
+                            if constexpr (kV8) {
+                                // 2 steps of 32 keys: P is 4 E4M3 per tensor-memory column, V rows are 128 B apart
+                                constexpr uint32_t idesc_pv8 = make_idesc_e4m3(128, 128);
 #pragma unroll
-                            for (int ks = 0; ks < BS / 16; ++ks)
-                                umma_ts(tOb, tPb + ks * 8, ((uint64_t)desc_hi << 32) | (vlo + (uint32_t)ks * (2048u >> 4)),
-                                        idesc_pv, (t >= 2 || ks > 0) ? 1u : 0u);
+                                for (int ks = 0; ks < 2; ++ks)
+                                    umma_ts_f8(tOb, tPb + ks * 8,
+                                               ((uint64_t)desc_hi << 32) | (vlo8 + (uint32_t)half * (8192u >> 4) + (uint32_t)ks * (4096u >> 4)),
+                                               idesc_pv8, ks > 0 ? 1u : first);
+                            } else {
+#pragma unroll
+                                for (int ks = 0; ks < 4; ++ks)
+                                    umma_ts(tOb, tPb + ks * 8,
+                                            ((uint64_t)desc_hi << 32) | (vlo + (uint32_t)half * (8192u >> 4) + (uint32_t)ks * (2048u >> 4)),
+                                            idesc_pv, ks > 0 ? 1u : first);
+                            }
+                            umma_commit(smem_u32(&sm.pv_done[b][half]));
+                            if (half == 1) umma_commit(smem_u32(&sm.v_empty[st]));
                         }
-                        umma_commit(smem_u32(&sm.v_empty[st]));
-                        umma_commit(smem_u32(&sm.pv_done[b]));
                         ++cnt;
                         ++ring;
                     }
@@ -406,33 +431,35 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             const int n_a = (c - a + 1) >> 1;     // blocks t = a, a + 2, ... of this stream
             float m_run = -INFINITY, l_run = 0.f;
 
-            for (int u = 0; u < n_a && ok; ++u) {
-                uint4 km = make_uint4(0xffffffffu, 0xffffffffu, 0xffffffffu, 0xffffffffu);
+            for (int v = 0; v < 2 * n_a && ok; ++v) {            // half-blocks of 64 keys of this stream
+                const int u = v >> 1, half = v & 1;
+                uint32_t kw0 = 0xffffffffu, kw1 = 0xffffffffu;    // validity of this half-block's 64 keys
                 if (has_pad) {
                     const int kb = min((int)irow[2 * u + a], m.nb - 1);
-                    km = __ldg(kmask + kb);
+                    const uint2 kv = __ldg(reinterpret_cast<const uint2*>(kmask + kb) + half);
+                    kw0 = kv.x;
+                    kw1 = kv.y;
                 }
-                ok = mbar_wait(smem_u32(&sm.s_full[a]), sn & 1u, abort_flag);
-                ++sn;
+                ok = mbar_wait(smem_u32(&sm.s_full[a][half]), (sn >> 1) & 1u, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
-                uint32_t s[128];
-#pragma unroll
-                for (int ch = 0; ch < 4; ++ch) tmem_ld32(tS + ch * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32 * ch]));
+                const uint32_t tSh = tS + 64u * half;
+                uint32_t s[64];
+                tmem_ld32(tSh, *reinterpret_cast<uint32_t(*)[32]>(&s[0]));
+                tmem_ld32(tSh + 32, *reinterpret_cast<uint32_t(*)[32]>(&s[32]));
                 tmem_wait_ld();
-                if ((km.x & km.y & km.z & km.w) != 0xffffffffu) {   // edge block: padded keys -> -inf
-                    const uint32_t kw[4] = {km.x, km.y, km.z, km.w};
+                if ((kw0 & kw1) != 0xffffffffu) {                 // edge block: padded keys -> -inf
 #pragma unroll
-                    for (int j = 0; j < 128; ++j)
-                        if (!((kw[j >> 5] >> (j & 31)) & 1u)) s[j] = 0xff800000u;
+                    for (int j = 0; j < 64; ++j)
+                        if (!(((j < 32 ? kw0 : kw1) >> (j & 31)) & 1u)) s[j] = 0xff800000u;
                 }
                 float mx0 = __uint_as_float(s[0]), mx1 = __uint_as_float(s[1]), mx2 = __uint_as_float(s[2]),
                       mx3 = __uint_as_float(s[3]);
 #pragma unroll
-                for (int j = 4; j < 128; j += 8) {
+                for (int j = 4; j < 64; j += 8) {
                     mx0 = max3(mx0, __uint_as_float(s[j]), __uint_as_float(s[j + 1]));
                     mx1 = max3(mx1, __uint_as_float(s[j + 2]), __uint_as_float(s[j + 3]));
-                    if (j + 4 < 128) {
+                    if (j + 4 < 64) {
                         mx2 = max3(mx2, __uint_as_float(s[j + 4]), __uint_as_float(s[j + 5]));
                         mx3 = max3(mx3, __uint_as_float(s[j + 6]), __uint_as_float(s[j + 7]));
                     }
@@ -447,7 +474,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         m_run = m_new;
                     }
                     l_run *= corr;
-                    if (u > 0) {
+                    if (v > 0) {
+                        // O still receives the previous half-block's P V: wait for that MMA before touching it
+                        ok = mbar_wait(smem_u32(&sm.pv_done[a][half ^ 1]), ((sn - 1u) >> 1) & 1u, abort_flag);
+                        if (!ok) break;
+                        tc_fence_after();
                         uint32_t r[32];
 #pragma unroll
                         for (int ch = 0; ch < 4; ++ch) {
@@ -462,9 +493,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 const float moff = (m_run == -INFINITY) ? 0.f : m_run * sl2;   // -inf only if no valid key yet
                 float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
                 if constexpr (kV8) {
-                    uint32_t pk8[32];                              // 4 E4M3 weights per column, lowest key in the lowest byte
+                    uint32_t pk8[16];                              // 4 E4M3 weights per column, lowest key in the lowest byte
 #pragma unroll
-                    for (int j = 0; j < 128; j += 4) {
+                    for (int j = 0; j < 64; j += 4) {
                         float e0 = __uint_as_float(s[j]), e1 = __uint_as_float(s[j + 1]), e2 = __uint_as_float(s[j + 2]),
                               e3 = __uint_as_float(s[j + 3]);
                         fma2(e0, e1, sl2, -moff);
@@ -476,11 +507,11 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         sum0 += p0; sum1 += p1; sum2 += p2; sum3 += p3;
                     }
                     l_run += (sum0 + sum1) + (sum2 + sum3);
-                    tmem_st32(tS, pk8);
+                    tmem_st16(tSh, pk8);
                 } else {
-                    uint32_t pk[64];
+                    uint32_t pk[32];
 #pragma unroll
-                    for (int j = 0; j < 128; j += 4) {
+                    for (int j = 0; j < 64; j += 4) {
                         float e0 = __uint_as_float(s[j]), e1 = __uint_as_float(s[j + 1]), e2 = __uint_as_float(s[j + 2]),
                               e3 = __uint_as_float(s[j + 3]);
                         fma2(e0, e1, sl2, -moff);
@@ -496,13 +527,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                         add_bf16_pair(sum2, sum3, whi);
                     }
                     l_run += (sum0 + sum1) + (sum2 + sum3);
-                    tmem_st32(tS, *reinterpret_cast<uint32_t(*)[32]>(&pk[0]));
-                    tmem_st32(tS + 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[32]));
+                    tmem_st32(tSh, pk);                           // P over the first 32 columns of this S slot
                 }
                 tmem_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&sm.p_full[a]));
+                if (lane == 0) mbar_arrive(smem_u32(&sm.p_full[a][half]));
+                ++sn;
             }
             if (!ok) break;
 
