@@ -5,8 +5,8 @@
 //   warp 0        producer: pops (head, query-block) tiles from the heaviest-first queue, TMA-loads
 //                 Q once per tile and the retained K tiles by index into a 3-deep ring
 //   warp 2        second producer: the retained V tiles into their own 3-deep ring
-//   warps 1, 3    MMA issuers (one thread each): warp 1 issues S = Q K^T, warp 3 issues O += P V, as
-//                 tcgen05 MMAs with the accumulators in tensor memory
+//   warps 1, 3    MMA issuers (one thread each), one per stream: S = Q K^T and O += P V as tcgen05
+//                 MMAs with the accumulators in tensor memory
 //   warps 4-7     softmax of the even retained blocks  (stream 0)
 //   warps 8-11    softmax of the odd retained blocks   (stream 1)
 // The retained blocks of a tile alternate between two independent streams, each with its own O
@@ -135,7 +135,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
     }
     if (tid == 0) {
         mbar_init(smem_u32(&sm.q_full), 1);
-        mbar_init(smem_u32(&sm.q_empty), 1);
+        mbar_init(smem_u32(&sm.q_empty), 2);
         for (int s = 0; s < KS; ++s) { mbar_init(smem_u32(&sm.k_full[s]), 1); mbar_init(smem_u32(&sm.k_empty[s]), 1); }
         for (int s = 0; s < VS; ++s) { mbar_init(smem_u32(&sm.v_full[s]), 1); mbar_init(smem_u32(&sm.v_empty[s]), 1); }
         for (int a = 0; a < 2; ++a)
@@ -144,7 +144,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 mbar_init(smem_u32(&sm.p_full[a][h]), 4);
                 mbar_init(smem_u32(&sm.pv_done[a][h]), 1);
             }
-        mbar_init(smem_u32(&sm.o_full), 1);
+        mbar_init(smem_u32(&sm.o_full), 2);
         mbar_init(smem_u32(&sm.o_free), 8);
         mbar_init(smem_u32(&sm.ml_ready), 8);
         mbar_init(smem_u32(&sm.ml_done), 8);
@@ -305,9 +305,32 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
             // S/P slots (one per half): the QK MMA of a stream's next half-block is finished while its softmax
             // warps are still on the current one, so in steady state they do not wait for the tensor pipe.
             constexpr uint32_t idesc_qk64 = make_idesc_bf16(128, 64, false);
-            uint32_t n = 0, ring = 0, qn = 0, cnt0 = 0, cnt1 = 0;   // cnt: blocks of each stream so far
+            // One issuer thread per stream (warp 1: stream 0, warp 3: stream 1).  Inside a stream the order
+            // PV(v), QK(v + 2) is program order, so the QK MMA that refills an S/P slot needs no barrier
+            // against the PV MMA that read it, and the stream's next half-block is on the tensor pipe as
+            // soon as the current P has been consumed; the two streams never wait on each other.
+            const int a = warp == 3 ? 1 : 0;
+            uint32_t n = 0, ring0 = 0, qn = 0, pcnt = 0;   // ring0: ring position of the tile's block 0; pcnt: half-blocks PV'd
             bool ok = true;
-            const bool is_qk = warp == 1;
+            const uint32_t tOa = tmem + kColO + 128u * a;
+
+            auto issue_qk = [&](int v) {                    // half-block v of this stream in the current tile
+                const int u = v >> 1, half = v & 1;
+                const uint32_t ring = ring0 + (uint32_t)(2 * u + a), st = ring % KS;
+                if (half == 0) ok = ok && mbar_wait(smem_u32(&sm.k_full[st]), (ring / KS) & 1u, abort_flag);
+                if (!ok) return;
+                tc_fence_after();
+                const uint32_t tSa = tmem + kColS + 128u * a + 64u * half;
+                const uint32_t kh = k_lo0 + st * (kTileBytes >> 4) + (uint32_t)half * (8192u >> 4);   // key rows 64 half ..
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off16 = ((uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u) >> 4;
+                    umma_ss(tSa, ((uint64_t)desc_hi << 32) | (q_lo + off16), ((uint64_t)desc_hi << 32) | (kh + off16), idesc_qk64,
+                            ks > 0 ? 1u : 0u);
+                }
+                if (half == 1) umma_commit(smem_u32(&sm.k_empty[st]));
+                umma_commit(smem_u32(&sm.s_full[a][half]));
+            };
 
             while (ok) {
                 const uint32_t slot = n % TS;
@@ -319,80 +342,58 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant_
                 ++n;
                 if (tile < 0) break;
                 if (c == 0) continue;
-                if (is_qk) {
-                    ok = mbar_wait(smem_u32(&sm.q_full), qn & 1u, abort_flag);
-                    for (int t = 0; t < c && ok; ++t) {
-                        const int a = t & 1;
-                        uint32_t& cnt = a ? cnt1 : cnt0;
-                        const uint32_t st = ring % KS, ph = (ring / KS) & 1u;
-                        ok = mbar_wait(smem_u32(&sm.k_full[st]), ph, abort_flag);
-                        const uint32_t klo = k_lo0 + st * (kTileBytes >> 4);
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            // the slot's previous occupant (this stream's previous block, same half) must have been
-                            // read by its PV
-                            if (ok && cnt > 0) ok = mbar_wait(smem_u32(&sm.pv_done[a][half]), (cnt - 1u) & 1u, abort_flag);
-                            if (!ok) break;
-                            tc_fence_after();
-                            const uint32_t tSa = tmem + kColS + 128u * a + 64u * half;
-                            const uint32_t kh = klo + (uint32_t)half * (8192u >> 4);        // key rows 64 half ..
-#pragma unroll
-                            for (int ks = 0; ks < D / 16; ++ks) {
-                                const uint32_t off16 = ((uint32_t)(ks >> 2) * kHalfBytes + (uint32_t)(ks & 3) * 32u) >> 4;
-                                umma_ss(tSa, ((uint64_t)desc_hi << 32) | (q_lo + off16), ((uint64_t)desc_hi << 32) | (kh + off16),
-                                        idesc_qk64, ks > 0 ? 1u : 0u);
-                            }
-                            if (half == 1) {
-                                umma_commit(smem_u32(&sm.k_empty[st]));
-                                if (t == c - 1) umma_commit(smem_u32(&sm.q_empty));
-                            }
-                            umma_commit(smem_u32(&sm.s_full[a][half]));
-                        }
-                        ++cnt;
-                        ++ring;
-                    }
-                } else {
-                    for (int t = 0; t < c && ok; ++t) {
-                        const int b = t & 1;
-                        uint32_t& cnt = b ? cnt1 : cnt0;
-                        const uint32_t st = ring % VS, ph = (ring / VS) & 1u;
-                        const uint32_t vlo = v_lo0 + st * (kTileBytes >> 4);
-                        const uint32_t vlo8 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.v[st]), 16, 1024);
-                        const uint32_t tOb = tmem + kColO + 128u * b;
-#pragma unroll
-                        for (int half = 0; half < 2; ++half) {
-                            ok = ok && mbar_wait(smem_u32(&sm.p_full[b][half]), cnt & 1u, abort_flag);
-                            if (half == 0) {
-                                ok = ok && mbar_wait(smem_u32(&sm.v_full[st]), ph, abort_flag);
-                                if (ok && t == 0) ok = mbar_wait(smem_u32(&sm.o_free), (qn & 1u) ^ 1u, abort_flag);
-                            }
-                            if (!ok) break;
-                            tc_fence_after();
-                            const uint32_t tPb = tmem + kColS + 128u * b + 64u * half;
-                            const uint32_t first = (t < 2 && half == 0) ? 0u : 1u;       // overwrite O on a stream's first half-block
-                            if constexpr (kV8) {
-                                // 2 steps of 32 keys: P is 4 E4M3 per tensor-memory column, V rows are 128 B apart
-                                constexpr uint32_t idesc_pv8 = make_idesc_e4m3(128, 128);
-#pragma unroll
-                                for (int ks = 0; ks < 2; ++ks)
-                                    umma_ts_f8(tOb, tPb + ks * 8,
-                                               ((uint64_t)desc_hi << 32) | (vlo8 + (uint32_t)half * (8192u >> 4) + (uint32_t)ks * (4096u >> 4)),
-                                               idesc_pv8, ks > 0 ? 1u : first);
-                            } else {
-#pragma unroll
-                                for (int ks = 0; ks < 4; ++ks)
-                                    umma_ts(tOb, tPb + ks * 8,
-                                            ((uint64_t)desc_hi << 32) | (vlo + (uint32_t)half * (8192u >> 4) + (uint32_t)ks * (2048u >> 4)),
-                                            idesc_pv, ks > 0 ? 1u : first);
-                            }
-                            umma_commit(smem_u32(&sm.pv_done[b][half]));
-                            if (half == 1) umma_commit(smem_u32(&sm.v_empty[st]));
-                        }
-                        ++cnt;
-                        ++ring;
-                    }
-                    if (ok) umma_commit(smem_u32(&sm.o_full));   // every PV done implies every QK done
+                const int n_a = (c - a + 1) >> 1, nv = 2 * n_a;
+                // Q loaded also means that the previous tile's q_empty phase is complete
+                ok = mbar_wait(smem_u32(&sm.q_full), qn & 1u, abort_flag);
+                if (ok && n_a == 0) {
+                    // c == 1 and this is stream 1: arrive in this tile's phases only
+                    ok = mbar_wait(smem_u32(&sm.o_free), (qn & 1u) ^ 1u, abort_flag);
+                    if (ok) { mbar_arrive(smem_u32(&sm.q_empty)); mbar_arrive(smem_u32(&sm.o_full)); }
                 }
+                if (ok && nv > 0) {
+                    issue_qk(0);
+                    issue_qk(1);
+                    if (ok && nv == 2) umma_commit(smem_u32(&sm.q_empty));     // this stream's last QK of the tile
+                }
+                for (int v = 0; v < nv && ok; ++v) {
+                    const int u = v >> 1, half = v & 1;
+                    const uint32_t ring = ring0 + (uint32_t)(2 * u + a), st = ring % VS;
+                    ok = mbar_wait(smem_u32(&sm.p_full[a][half]), (pcnt >> 1) & 1u, abort_flag);
+                    if (half == 0) {
+                        ok = ok && mbar_wait(smem_u32(&sm.v_full[st]), (ring / VS) & 1u, abort_flag);
+                        if (ok && v == 0) ok = mbar_wait(smem_u32(&sm.o_free), (qn & 1u) ^ 1u, abort_flag);
+                    }
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t tPb = tmem + kColS + 128u * a + 64u * half;
+                    const uint32_t first = v == 0 ? 0u : 1u;                   // overwrite O on a stream's first half-block
+                    if constexpr (kV8) {
+                        // 2 steps of 32 keys: P is 4 E4M3 per tensor-memory column, V rows are 128 B apart
+                        constexpr uint32_t idesc_pv8 = make_idesc_e4m3(128, 128);
+                        const uint32_t vlo8 = (uint32_t)make_smem_desc_sw128(smem_u32(sm.v[st]), 16, 1024);
+#pragma unroll
+                        for (int ks = 0; ks < 2; ++ks)
+                            umma_ts_f8(tOa, tPb + ks * 8,
+                                       ((uint64_t)desc_hi << 32) | (vlo8 + (uint32_t)half * (8192u >> 4) + (uint32_t)ks * (4096u >> 4)),
+                                       idesc_pv8, ks > 0 ? 1u : first);
+                    } else {
+                        const uint32_t vlo = v_lo0 + st * (kTileBytes >> 4);
+#pragma unroll
+                        for (int ks = 0; ks < 4; ++ks)
+                            umma_ts(tOa, tPb + ks * 8,
+                                    ((uint64_t)desc_hi << 32) | (vlo + (uint32_t)half * (8192u >> 4) + (uint32_t)ks * (2048u >> 4)),
+                                    idesc_pv, ks > 0 ? 1u : first);
+                    }
+                    umma_commit(smem_u32(&sm.pv_done[a][half]));             // for the softmax warps' rare rescale of O
+                    if (half == 1) umma_commit(smem_u32(&sm.v_empty[st]));
+                    ++pcnt;
+                    if (v + 2 < nv) {
+                        issue_qk(v + 2);                                       // refills the slot PV(v) has just read
+                        if (ok && v + 3 == nv) umma_commit(smem_u32(&sm.q_empty));   // that was the stream's last QK of the tile
+                    }
+                }
+                if (ok && nv > 0) umma_commit(smem_u32(&sm.o_full));          // this stream's PVs (hence its QKs) are done
+                ring0 += (uint32_t)c;
                 ++qn;
             }
             failed = !ok;
